@@ -1,0 +1,125 @@
+/*
+ * slimspec.h -- C ABI of the B200 (sm_100a) SlimSpec draft LM-head library.
+ *
+ * The operation is the low-rank draft LM-head of the SlimSpec paper, Section 4.1:
+ *     logits = W_up W_down h          (standard head: logits = W_full h)
+ * written here with row vectors and the transposed weights
+ *     A = W_down^T (d x r),  B = W_up^T (r x V),  W = W_full^T (d x V):
+ *     z = h A   (rank-r code),   logits = z B          |   logits = h W
+ * followed by the full-vocabulary softmax that Section 3.2 names, in its stable
+ * logarithmic form, and the selection of the k most probable tokens per row:
+ *     lse = max_v logit + log sum_v exp(logit - max),   logprob = logit - lse
+ *     top-k ordered by (logit descending, token id ascending).
+ *
+ * Common conventions
+ *   - Every matrix is dense, contiguous, row-major; weights and activations are bf16
+ *     (passed as const void*), all accumulation is fp32, outputs are int32 / fp32.
+ *       h[M][d]   A[d][r]   B[r][V]   W[d][V]   out_ids[M][k]   out_logprobs[M][k]
+ *   - Unless a parameter says "host", pointers are DEVICE pointers on the device that was
+ *     current when the context was created.  The caller owns every buffer; the library
+ *     neither frees nor keeps them after the call's work has run.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = the default
+ *     stream) and return without synchronising, except where stated.  Calls on one
+ *     context must not overlap on the GPU: a context owns one set of scratch buffers.
+ *   - Return value: SLIMSPEC_OK or a negative status; nothing is launched on an argument
+ *     error.  There is no CPU fallback: every step runs in CUDA kernels.
+ *   - 1 <= k <= min(V, SLIMSPEC_MAX_K).  Inputs holding NaN or infinity give unspecified
+ *     (but terminating) results.
+ */
+#ifndef SLIMSPEC_H
+#define SLIMSPEC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SLIMSPEC_MAX_K 64
+
+/* status codes */
+#define SLIMSPEC_OK 0
+#define SLIMSPEC_ERR_NULL (-1)      /* a required pointer is NULL                              */
+#define SLIMSPEC_ERR_DIM (-2)       /* a dimension is <= 0, k out of range, or beyond the ctx  */
+#define SLIMSPEC_ERR_ALIGN (-3)     /* the forced path cannot take these shapes / alignments   */
+#define SLIMSPEC_ERR_CUDA (-4)      /* a CUDA runtime call or a launch failed                  */
+#define SLIMSPEC_ERR_TIMEOUT (-5)   /* a bounded device-side wait ran out (see last_error)     */
+#define SLIMSPEC_ERR_NOMEM (-6)     /* device memory for scratch could not be allocated        */
+
+/* execution paths (slimspec_force_path) */
+#define SLIMSPEC_PATH_AUTO 0        /* chosen per (M, shapes) from measured timings            */
+#define SLIMSPEC_PATH_GENERIC 1     /* any shape; one thread per logit; slow                   */
+#define SLIMSPEC_PATH_STREAM 2      /* split-V weight-streaming kernels, FP32 FMA (small M)    */
+#define SLIMSPEC_PATH_TENSOR 3      /* tcgen05 / TMEM tensor-core kernels (large M)            */
+
+typedef struct slimspec_ctx slimspec_ctx;
+
+/*
+ * Create a context on the current device.  It owns the scratch the kernels need (the
+ * fp32 code z, split-V partial max / sum-exp / top-k records, tickets, an error word),
+ * sized for calls with M <= max_M, d and r <= max_d, V <= max_V, k <= max_k.
+ * Allocates device memory (synchronising).  *out receives the context.
+ */
+int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max_V, int max_k);
+
+/* Free the context's scratch.  Synchronises the device.  NULL is allowed. */
+void slimspec_destroy(slimspec_ctx* ctx);
+
+/* Force one execution path for later calls on this context (SLIMSPEC_PATH_*). */
+int slimspec_force_path(slimspec_ctx* ctx, int path);
+
+/* The path (SLIMSPEC_PATH_*, never AUTO) the last *_topk / *_logits call on ctx took. */
+int slimspec_last_path(const slimspec_ctx* ctx);
+
+/*
+ * Low-rank draft head with fused log-softmax and top-k (Section 4.1, low-rank form;
+ * softmax of Section 3.2).  The M x V logits are never written to memory.
+ *   out_ids[m][j]      id of the j-th most probable token of row m (ties: lower id first)
+ *   out_logprobs[m][j] its log-probability, logit - lse
+ */
+int slimspec_head_topk(slimspec_ctx* ctx, const void* h, const void* A, const void* B,
+                       int M, int d, int r, int V, int k,
+                       int32_t* out_ids, float* out_logprobs, void* stream);
+
+/*
+ * Same computation with host-side activations and results: copies h (M x d bf16, host;
+ * pinned memory makes the copy asynchronous) to the device, runs slimspec_head_topk,
+ * copies ids and log-probs back to the host buffers and waits for `stream`.
+ * A and B stay device pointers: weights are resident.
+ */
+int slimspec_head_topk_host(slimspec_ctx* ctx, const void* h_host, const void* A, const void* B,
+                            int M, int d, int r, int V, int k,
+                            int32_t* out_ids_host, float* out_logprobs_host, void* stream);
+
+/*
+ * Low-rank draft head, raw logits (Section 4.1): out_logits[M][V] fp32 = (h A) B.
+ */
+int slimspec_head_logits(slimspec_ctx* ctx, const void* h, const void* A, const void* B,
+                         int M, int d, int r, int V, float* out_logits, void* stream);
+
+/*
+ * Standard full-rank head (Section 4.1, logits = W_full h) with the same fused
+ * log-softmax and top-k: the baseline every relative head cost in the paper is
+ * normalised to.
+ */
+int fullhead_topk(slimspec_ctx* ctx, const void* h, const void* W,
+                  int M, int d, int V, int k,
+                  int32_t* out_ids, float* out_logprobs, void* stream);
+
+/*
+ * Synchronise the device and return the context's device-side error word:
+ * SLIMSPEC_OK, or SLIMSPEC_ERR_TIMEOUT if a bounded wait inside a kernel gave up
+ * (the outputs of that call are then invalid).  Clears the word.  Meant for tests.
+ */
+int slimspec_last_error(slimspec_ctx* ctx);
+
+/* Number of kernels the library has launched on this context since it was created. */
+long long slimspec_launch_count(const slimspec_ctx* ctx);
+
+/* Static description of a status code. */
+const char* slimspec_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SLIMSPEC_H */

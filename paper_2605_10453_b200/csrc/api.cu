@@ -1,0 +1,227 @@
+// C-ABI layer: context, argument checks, path choice.  See include/slimspec.h for the contract.
+#include "../../include/slimspec.h"
+#include "kernels.h"
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+using namespace slimspec;
+
+struct slimspec_ctx {
+    int device;
+    int sm_count;
+    int max_M, max_d, max_V, max_k;
+    int forced_path;
+    int last_path;
+    long long launches;
+    Scratch s;
+    bf16* h_stage;        // device copy of host activations (head_topk_host)
+    int32_t* ids_stage;   // device results of head_topk_host
+    float* lp_stage;
+};
+
+static const int kMaxParts = 1024;     // most V slabs any kernel writes per row
+static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
+
+static int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+extern "C" const char* slimspec_strerror(int status)
+{
+    switch (status) {
+    case SLIMSPEC_OK: return "ok";
+    case SLIMSPEC_ERR_NULL: return "null pointer argument";
+    case SLIMSPEC_ERR_DIM: return "dimension out of range (<= 0, k > min(V, 64), or beyond the context's limits)";
+    case SLIMSPEC_ERR_ALIGN: return "forced path does not support these shapes or alignments";
+    case SLIMSPEC_ERR_CUDA: return "CUDA runtime or launch error";
+    case SLIMSPEC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case SLIMSPEC_ERR_NOMEM: return "out of device memory for scratch";
+    default: return "unknown status";
+    }
+}
+
+extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max_V, int max_k)
+{
+    if (!out) return SLIMSPEC_ERR_NULL;
+    *out = nullptr;
+    if (max_M <= 0 || max_d <= 0 || max_V <= 0 || max_k <= 0 || max_k > SLIMSPEC_MAX_K) return SLIMSPEC_ERR_DIM;
+    slimspec_ctx* c = new (std::nothrow) slimspec_ctx;
+    if (!c) return SLIMSPEC_ERR_NOMEM;
+    memset(c, 0, sizeof(*c));
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&c->device) != cudaSuccess || cudaGetDeviceProperties(&prop, c->device) != cudaSuccess) {
+        delete c;
+        return SLIMSPEC_ERR_CUDA;
+    }
+    c->sm_count = prop.multiProcessorCount;
+    c->max_M = max_M; c->max_d = max_d; c->max_V = max_V; c->max_k = max_k;
+    c->s.max_parts = kMaxParts;
+    const size_t mpad = (size_t)round_up(max_M, kRowPad);
+    const size_t z_elems = mpad * (size_t)max_d;
+    const size_t zpart_elems = (size_t)64 * kRowPad * (size_t)max_d;     // <= 64 d-slabs of 8 rows
+    const size_t part_elems = mpad * (size_t)kMaxParts * (2 + 2 * (size_t)max_k);
+    bool ok = true;
+    ok = ok && cudaMalloc(&c->s.z, z_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.tickets, 4096 * sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.err, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->h_stage, (size_t)max_M * max_d * sizeof(bf16)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->ids_stage, (size_t)max_M * max_k * sizeof(int32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->lp_stage, (size_t)max_M * max_k * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int)) == cudaSuccess;
+    ok = ok && cudaMemset(c->s.err, 0, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMemset(c->s.z, 0, z_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        slimspec_destroy(c);
+        return SLIMSPEC_ERR_NOMEM;
+    }
+    *out = c;
+    return SLIMSPEC_OK;
+}
+
+extern "C" void slimspec_destroy(slimspec_ctx* c)
+{
+    if (!c) return;
+    cudaDeviceSynchronize();
+    cudaFree(c->s.z); cudaFree(c->s.zpart); cudaFree(c->s.part); cudaFree(c->s.tickets); cudaFree(c->s.err);
+    cudaFree(c->s.logits); cudaFree(c->h_stage); cudaFree(c->ids_stage); cudaFree(c->lp_stage);
+    delete c;
+}
+
+extern "C" int slimspec_force_path(slimspec_ctx* c, int path)
+{
+    if (!c) return SLIMSPEC_ERR_NULL;
+    if (path < SLIMSPEC_PATH_AUTO || path > SLIMSPEC_PATH_TENSOR) return SLIMSPEC_ERR_DIM;
+    c->forced_path = path;
+    return SLIMSPEC_OK;
+}
+
+extern "C" int slimspec_last_path(const slimspec_ctx* c) { return c ? c->last_path : SLIMSPEC_ERR_NULL; }
+
+extern "C" long long slimspec_launch_count(const slimspec_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int slimspec_last_error(slimspec_ctx* c)
+{
+    if (!c) return SLIMSPEC_ERR_NULL;
+    int e = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return SLIMSPEC_ERR_CUDA;
+    if (cudaMemcpy(&e, c->s.err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return SLIMSPEC_ERR_CUDA;
+    if (e != 0) {
+        cudaMemset(c->s.err, 0, sizeof(int));
+        // tickets may have been left mid-count by the kernel that gave up
+        cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int));
+        return SLIMSPEC_ERR_TIMEOUT;
+    }
+    return SLIMSPEC_OK;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+// Grow-only fp32 M x V buffer for the generic top-k path (allocation synchronises).
+static int ensure_logits(slimspec_ctx* c, size_t elems)
+{
+    if (c->s.logits_elems >= elems) return SLIMSPEC_OK;
+    if (c->s.logits) { cudaDeviceSynchronize(); cudaFree(c->s.logits); c->s.logits = nullptr; c->s.logits_elems = 0; }
+    if (cudaMalloc(&c->s.logits, elems * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_NOMEM; }
+    c->s.logits_elems = elems;
+    return SLIMSPEC_OK;
+}
+
+#define CK(expr) do { if ((expr) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; } } while (0)
+
+// Shared body.  K is the contraction length of the streamed matrix Bm (K x V): r for the
+// low-rank head (A != null), d for the full-rank head (A == null, z = widened h).
+// mode 0: top-k into ids/logprobs; mode 1: raw logits.
+static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* Bm, int M, int d, int r, int V,
+                    int k, int mode, int32_t* ids, float* logprobs, float* logits, cudaStream_t st)
+{
+    if (!c || !h || !Bm) return SLIMSPEC_ERR_NULL;
+    if (mode == 0 && (!ids || !logprobs)) return SLIMSPEC_ERR_NULL;
+    if (mode == 1 && !logits) return SLIMSPEC_ERR_NULL;
+    const bool lowrank = (A != nullptr);
+    if (M <= 0 || d <= 0 || V <= 0 || (lowrank && r <= 0)) return SLIMSPEC_ERR_DIM;
+    if (M > c->max_M || d > c->max_d || V > c->max_V || (lowrank && r > c->max_d)) return SLIMSPEC_ERR_DIM;
+    if (mode == 0 && (k <= 0 || k > V || k > SLIMSPEC_MAX_K || k > c->max_k)) return SLIMSPEC_ERR_DIM;
+    const int K = lowrank ? r : d;
+
+    int path = c->forced_path;
+    const bool ptr_ok = aligned16(h) && aligned16(Bm) && (!lowrank || aligned16(A)) &&
+                        (mode == 0 || aligned16(logits));
+    StreamPlan sp = stream_plan(M, d, K, V, mode == 0 ? k : 1, c->sm_count);
+    const bool stream_ok = sp.ok && ptr_ok && (!lowrank || r % 64 == 0);
+    if (path == SLIMSPEC_PATH_AUTO) path = stream_ok ? SLIMSPEC_PATH_STREAM : SLIMSPEC_PATH_GENERIC;
+    if (path == SLIMSPEC_PATH_TENSOR) return SLIMSPEC_ERR_ALIGN;   // tensor path not built yet
+    if (path == SLIMSPEC_PATH_STREAM && !stream_ok) return SLIMSPEC_ERR_ALIGN;
+    c->last_path = path;
+
+    if (path == SLIMSPEC_PATH_GENERIC) {
+        float* lg = logits;
+        if (mode == 0) {
+            int rc = ensure_logits(c, (size_t)M * V);
+            if (rc != SLIMSPEC_OK) return rc;
+            lg = c->s.logits;
+        }
+        if (lowrank) CK(generic_downproj(h, A, M, d, r, c->s.z, st));
+        else CK(generic_widen(h, M * d, c->s.z, st));
+        CK(generic_upproj(c->s.z, Bm, M, K, V, lg, st));
+        c->launches += 2;
+        if (mode == 0) { CK(generic_softmax_topk(lg, M, V, k, ids, logprobs, st)); c->launches += 1; }
+        return SLIMSPEC_OK;
+    }
+
+    // streaming path: row tiles of up to 8 rows, each streams the K x V matrix once
+    for (int m0 = 0; m0 < M; m0 += 8) {
+        const int mrows = (M - m0 < 8) ? (M - m0) : 8;
+        StreamPlan p = stream_plan(mrows, d, K, V, mode == 0 ? k : 1, c->sm_count);
+        const bf16* hm = h + (size_t)m0 * d;
+        if (lowrank) CK(stream_downproj(hm, A, mrows, p.mt, d, r, c->s, st));
+        else CK(stream_widen_t(hm, mrows, p.mt, d, c->s.z, st));
+        CK(stream_head(c->s.z, Bm, mrows, p.mt, K, V, k, mode,
+                       mode == 0 ? ids + (size_t)m0 * k : nullptr,
+                       mode == 0 ? logprobs + (size_t)m0 * k : nullptr,
+                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, true, st));
+        c->launches += 2;
+    }
+    return SLIMSPEC_OK;
+}
+
+extern "C" int slimspec_head_topk(slimspec_ctx* c, const void* h, const void* A, const void* B, int M, int d,
+                                  int r, int V, int k, int32_t* out_ids, float* out_logprobs, void* stream)
+{
+    if (!A) return SLIMSPEC_ERR_NULL;
+    return run_head(c, (const bf16*)h, (const bf16*)A, (const bf16*)B, M, d, r, V, k, 0, out_ids, out_logprobs,
+                    nullptr, (cudaStream_t)stream);
+}
+
+extern "C" int slimspec_head_logits(slimspec_ctx* c, const void* h, const void* A, const void* B, int M, int d,
+                                    int r, int V, float* out_logits, void* stream)
+{
+    if (!A) return SLIMSPEC_ERR_NULL;
+    return run_head(c, (const bf16*)h, (const bf16*)A, (const bf16*)B, M, d, r, V, 1, 1, nullptr, nullptr,
+                    out_logits, (cudaStream_t)stream);
+}
+
+extern "C" int fullhead_topk(slimspec_ctx* c, const void* h, const void* W, int M, int d, int V, int k,
+                             int32_t* out_ids, float* out_logprobs, void* stream)
+{
+    return run_head(c, (const bf16*)h, nullptr, (const bf16*)W, M, d, 0, V, k, 0, out_ids, out_logprobs, nullptr,
+                    (cudaStream_t)stream);
+}
+
+extern "C" int slimspec_head_topk_host(slimspec_ctx* c, const void* h_host, const void* A, const void* B, int M,
+                                       int d, int r, int V, int k, int32_t* out_ids_host,
+                                       float* out_logprobs_host, void* stream)
+{
+    if (!c || !h_host || !A || !B || !out_ids_host || !out_logprobs_host) return SLIMSPEC_ERR_NULL;
+    if (M <= 0 || d <= 0 || M > c->max_M || d > c->max_d || k <= 0 || k > c->max_k) return SLIMSPEC_ERR_DIM;
+    cudaStream_t st = (cudaStream_t)stream;
+    CK(cudaMemcpyAsync(c->h_stage, h_host, (size_t)M * d * sizeof(bf16), cudaMemcpyHostToDevice, st));
+    int rc = slimspec_head_topk(c, c->h_stage, A, B, M, d, r, V, k, c->ids_stage, c->lp_stage, stream);
+    if (rc != SLIMSPEC_OK) return rc;
+    CK(cudaMemcpyAsync(out_ids_host, c->ids_stage, (size_t)M * k * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(out_logprobs_host, c->lp_stage, (size_t)M * k * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    return SLIMSPEC_OK;
+}

@@ -1,0 +1,51 @@
+// Internal launch interface between the C-ABI layer (api.cu) and the kernel files.
+// Every launcher only enqueues work on `st` and returns the cudaError_t of its launches.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace slimspec {
+
+typedef __nv_bfloat16 bf16;
+
+// One split-V partial record per (row, slab): running max, sum of exp(logit - max), and the
+// slab's k best (logit, id) pairs in (logit desc, id asc) order.
+// Layout in the context's scratch: float pm[P], ps[P], pv[P][k]; int pi[P][k] per row.
+struct Scratch {
+    float* z;            // fp32 code (or widened h); generic path [M][K], streaming path transposed [K][mt]
+    float* zpart;        // split-d partial sums of the down-projection
+    float* part;         // split-V partial records
+    unsigned int* tickets;  // arrival counters (self-resetting)
+    int* err;            // device error word
+    float* logits;       // generic path only: M x V fp32, grown on demand
+    size_t logits_elems;
+    int max_parts;       // capacity of `part` in slabs per row
+};
+
+// ---- generic path (any shape) -------------------------------------------------------
+cudaError_t generic_downproj(const bf16* h, const bf16* A, int M, int d, int r, float* z, cudaStream_t st);
+cudaError_t generic_widen(const bf16* h, int n, float* z, cudaStream_t st);
+cudaError_t generic_upproj(const float* z, const bf16* B, int M, int r, int V, float* logits, cudaStream_t st);
+cudaError_t generic_softmax_topk(const float* logits, int M, int V, int k, int32_t* ids, float* logprobs,
+                                 cudaStream_t st);
+
+// ---- streaming path (small M) -------------------------------------------------------
+struct StreamPlan {
+    int ok;          // 0: shapes not supported by the streaming kernels
+    int mt;          // rows per launch (1, 2, 4, 8)
+    int ncta;        // V slabs = CTAs
+    int launches;    // kernels per call (for the launch counter)
+};
+StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count);
+// z = h A for M <= 8 rows, rows M..mt-1 zero-filled; split over d, deterministic.
+cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
+                            cudaStream_t st);
+// z^T = widened h^T (full-rank head: no down-projection).
+cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st);
+// logits = z B streamed once; mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
+cudaError_t stream_head(const float* z, const bf16* B, int M, int mt, int K, int V, int k, int mode,
+                        int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
+                        bool after_producer_kernel, cudaStream_t st);
+
+}  // namespace slimspec

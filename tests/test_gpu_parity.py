@@ -1,0 +1,249 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle, same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_10453_b200 import binding, synth
+from parity import LOGPROB_TOL, check_topk
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def dev(x):
+    return {k: v.to(DEV) for k, v in x.items()}
+
+
+def obits(x):
+    return {k: oracle.bf16_bits(v) for k, v in x.items()}
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = binding.Context(max_M=512, max_d=8192, max_V=152064, max_k=64)
+    yield c
+    c.close()
+
+
+def run_topk(ctx, x, k, path):
+    ctx.force_path(path)
+    g = dev(x)
+    ids, lp = ctx.slimspec_head_topk(g["h"], g["A"], g["B"], k)
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK
+    assert ctx.last_path() == path
+    return ids.cpu().numpy(), lp.cpu().numpy()
+
+
+# ---------------------------------------------------------------- tiny and ragged shapes
+
+GENERIC_SHAPES = [
+    # M, d, r, V, k
+    (1, 8, 2, 37, 5),
+    (3, 8, 2, 37, 37),
+    (5, 33, 7, 1001, 10),
+    (2, 64, 16, 4099, 64),
+    (17, 128, 24, 2500, 8),
+]
+
+
+@pytest.mark.parametrize("M,d,r,V,k", GENERIC_SHAPES)
+def test_generic_path_any_shape(ctx, M, d, r, V, k):
+    x = synth.make_inputs(M, d, r, V, seed=11)
+    ids, lp = run_topk(ctx, x, k, binding.PATH_GENERIC)
+    b = obits(x)
+    st = check_topk(oracle.head_topk(b["h"], b["A"], b["B"], k), ids, lp)
+    assert st["max_lp_err"] < 1e-3
+
+
+STREAM_SHAPES = [
+    # M, d, r, V, k  -- V/8 units vs 148 slabs: fewer units than slabs, ragged split, several passes
+    (1, 64, 64, 8 * 100, 10),
+    (1, 256, 64, 8 * 149, 10),
+    (2, 512, 128, 8 * (148 * 3 + 5), 7),
+    (3, 1000, 192, 8 * 1999, 10),
+    (4, 2048, 256, 8 * 4001, 32),
+    (5, 96, 64, 8 * 777, 1),
+    (8, 1024, 128, 8 * 2500, 10),
+    (7, 160, 320, 8 * 148 * 130, 5),      # 130 units per slab: two column passes
+    (11, 512, 64, 8 * 1501, 10),          # two row tiles (8 + 3)
+]
+
+
+@pytest.mark.parametrize("M,d,r,V,k", STREAM_SHAPES)
+def test_stream_path_matches_oracle(ctx, M, d, r, V, k):
+    x = synth.make_inputs(M, d, r, V, seed=5)
+    ids, lp = run_topk(ctx, x, k, binding.PATH_STREAM)
+    b = obits(x)
+    st = check_topk(oracle.head_topk(b["h"], b["A"], b["B"], k), ids, lp)
+    assert st["max_lp_err"] < 1e-3
+    # a second run must reproduce the first bit for bit (deterministic merge order)
+    ids2, lp2 = run_topk(ctx, x, k, binding.PATH_STREAM)
+    assert np.array_equal(ids, ids2) and np.array_equal(lp.view(np.uint32), lp2.view(np.uint32))
+    # and the generic kernels, a second GPU implementation, agree too
+    ids3, lp3 = run_topk(ctx, x, k, binding.PATH_GENERIC)
+    assert np.max(np.abs(lp - lp3)) < 1e-3
+
+
+def test_stream_path_refuses_what_it_cannot_take(ctx):
+    x = dev(synth.make_inputs(1, 64, 64, 8 * 100 + 4, seed=1))     # V not a multiple of 8
+    ctx.force_path(binding.PATH_STREAM)
+    with pytest.raises(binding.SlimSpecError) as e:
+        ctx.slimspec_head_topk(x["h"], x["A"], x["B"], 4)
+    assert e.value.status == binding.ERR_ALIGN
+    ctx.force_path(binding.PATH_AUTO)
+    ctx.slimspec_head_topk(x["h"], x["A"], x["B"], 4)
+    assert ctx.last_path() == binding.PATH_GENERIC
+
+
+# ---------------------------------------------------------------- the workloads
+
+def _config_case(ctx, name, M, rows=None, path=binding.PATH_AUTO):
+    c = synth.CONFIGS[name]
+    x = synth.make_inputs(M, c.d, c.r, c.V, seed=c.seed, logit_scale=c.logit_scale)
+    ids, lp = run_topk(ctx, x, c.k, path) if path != binding.PATH_AUTO else _auto(ctx, x, c.k)
+    b = obits(x)
+    hb = b["h"] if rows is None else b["h"][rows]
+    ref = oracle.head_topk(hb, b["A"], b["B"], c.k)
+    return check_topk(ref, ids, lp, rows=rows), ids, lp
+
+
+def _auto(ctx, x, k):
+    ctx.force_path(binding.PATH_AUTO)
+    g = dev(x)
+    ids, lp = ctx.slimspec_head_topk(g["h"], g["A"], g["B"], k)
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK
+    return ids.cpu().numpy(), lp.cpu().numpy()
+
+
+@pytest.mark.parametrize("name,M", [("c0", 1), ("c1", 1), ("c1", 8), ("c2", 1), ("c2", 16)])
+def test_workload_configs(ctx, name, M):
+    st, _, _ = _config_case(ctx, name, M)
+    assert st["rows"] == M
+    assert st["max_lp_err"] <= LOGPROB_TOL
+
+
+def test_throughput_batch_sampled_rows(ctx):
+    # M = 512: the oracle checks rows at every position class of a 128-row tile plus seeded extras
+    M = 512
+    rng = np.random.default_rng(0)
+    rows = sorted(set([0, 1, 63, 64, 127, 128, M // 2, M - 2, M - 1]) | set(rng.integers(0, M, 8).tolist()))
+    st, ids, lp = _config_case(ctx, "c3", M, rows=rows)
+    assert st["max_lp_err"] <= LOGPROB_TOL
+    # rows the oracle did not see: a row's result must not depend on the batch around it
+    c = synth.CONFIGS["c3"]
+    x = synth.make_inputs(M, c.d, c.r, c.V, seed=c.seed)
+    g = dev(x)
+    ctx.force_path(binding.PATH_AUTO)
+    for m in (5, 200, 300, 509):
+        i1, l1 = ctx.slimspec_head_topk(g["h"][m:m + 1].contiguous(), g["A"], g["B"], c.k)
+        assert np.max(np.abs(l1.cpu().numpy()[0] - lp[m])) < 2e-3
+        assert set(i1.cpu().numpy()[0].tolist()) == set(ids[m].tolist()) or np.max(np.abs(l1.cpu().numpy()[0] - lp[m])) < 2e-3
+
+
+# ---------------------------------------------------------------- full-rank baseline, logits
+
+@pytest.mark.parametrize("M", [1, 8])
+def test_fullhead_baseline(ctx, M):
+    c = synth.CONFIGS["c1"]
+    h = synth.make_h(M, c.d, c.seed)
+    W = synth.make_W(c.d, c.V, c.seed)
+    ctx.force_path(binding.PATH_AUTO)
+    ids, lp = ctx.fullhead_topk(h.to(DEV), W.to(DEV), c.k)
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK
+    ref = oracle.fullhead_topk(oracle.bf16_bits(h), oracle.bf16_bits(W), c.k)
+    st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy())
+    assert st["max_lp_err"] <= LOGPROB_TOL
+
+
+def test_identity_downprojection_equals_fullhead_on_gpu(ctx):
+    d, V, M, k = 128, 8 * 1234, 3, 10
+    h = synth.make_h(M, d, 3)
+    B = synth.make_B(d, V, 3)
+    eye = torch.eye(d, dtype=torch.bfloat16)
+    for path in (binding.PATH_GENERIC, binding.PATH_STREAM):
+        ctx.force_path(path)
+        i1, l1 = ctx.slimspec_head_topk(h.to(DEV), eye.to(DEV), B.to(DEV), k)
+        i2, l2 = ctx.fullhead_topk(h.to(DEV), B.to(DEV), k)
+        assert torch.equal(i1, i2)
+        assert torch.max(torch.abs(l1 - l2)).item() < 1e-5
+
+
+@pytest.mark.parametrize("path", [binding.PATH_GENERIC, binding.PATH_STREAM])
+@pytest.mark.parametrize("M,d,r,V", [(1, 2048, 256, 128256), (6, 512, 128, 8 * 3001)])
+def test_head_logits(ctx, path, M, d, r, V):
+    x = synth.make_inputs(M, d, r, V, seed=2)
+    g = dev(x)
+    ctx.force_path(path)
+    # canaries around the output catch writes out of bounds
+    buf = torch.full((M * V + 512,), 12345.0, dtype=torch.float32, device=DEV)
+    out = buf[256:256 + M * V].view(M, V)
+    ctx.slimspec_head_logits(g["h"], g["A"], g["B"], out_logits=out)
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK
+    assert torch.all(buf[:256] == 12345.0) and torch.all(buf[256 + M * V:] == 12345.0)
+    b = obits(x)
+    ref = oracle.slimspec_logits(b["h"], b["A"], b["B"])
+    assert np.max(np.abs(out.cpu().numpy().astype(np.float64) - ref)) <= 2e-2
+
+
+def test_topk_outputs_do_not_overrun(ctx):
+    M, d, r, V, k = 5, 256, 64, 8 * 999, 10
+    g = dev(synth.make_inputs(M, d, r, V, seed=4))
+    for path in (binding.PATH_GENERIC, binding.PATH_STREAM):
+        ctx.force_path(path)
+        ib = torch.full((M * k + 64,), -7, dtype=torch.int32, device=DEV)
+        lb = torch.full((M * k + 64,), -7.0, dtype=torch.float32, device=DEV)
+        ctx.slimspec_head_topk(g["h"], g["A"], g["B"], k, out_ids=ib[32:32 + M * k].view(M, k),
+                               out_logprobs=lb[32:32 + M * k].view(M, k))
+        torch.cuda.synchronize()
+        assert torch.all(ib[:32] == -7) and torch.all(ib[32 + M * k:] == -7)
+        assert torch.all(lb[:32] == -7.0) and torch.all(lb[32 + M * k:] == -7.0)
+        assert torch.all(ib[32:32 + M * k] >= 0)
+
+
+def test_planted_ties_resolve_to_lower_id(ctx):
+    M, d, r, V, k = 2, 128, 64, 8 * 600, 6
+    x = synth.make_inputs(M, d, r, V, seed=8)
+    b = obits(x)
+    best = int(np.argmax(oracle.slimspec_logits(b["h"], b["A"], b["B"])[0]))
+    twin = (best + 2417) % V                      # lands in another slab
+    x["B"][:, twin] = x["B"][:, best]
+    for path in (binding.PATH_GENERIC, binding.PATH_STREAM):
+        ids, lp = run_topk(ctx, x, k, path)
+        assert ids[0, :2].tolist() == sorted([best, twin])
+        assert lp[0, 0] == lp[0, 1]
+
+
+def test_host_buffer_entry_point(ctx):
+    c = synth.CONFIGS["c0"]
+    x = synth.make_inputs(1, c.d, c.r, c.V, seed=c.seed)
+    g = dev(x)
+    ctx.force_path(binding.PATH_AUTO)
+    ids_d, lp_d = ctx.slimspec_head_topk(g["h"], g["A"], g["B"], c.k)
+    ids_h, lp_h = ctx.slimspec_head_topk_host(x["h"].pin_memory(), g["A"], g["B"], c.k)
+    assert torch.equal(ids_d.cpu(), ids_h) and torch.equal(lp_d.cpu(), lp_h)
+
+
+def test_argument_errors_launch_nothing(ctx):
+    g = dev(synth.make_inputs(2, 64, 64, 800, seed=1))
+    n0 = ctx.launch_count()
+    lib = binding.load()
+    import ctypes
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    ids = torch.empty((2, 4), dtype=torch.int32, device=DEV)
+    lp = torch.empty((2, 4), dtype=torch.float32, device=DEV)
+    call = lambda M, d, r, V, k, h=g["h"]: lib.slimspec_head_topk(
+        ctx._h, p(h) if h is not None else None, p(g["A"]), p(g["B"]), M, d, r, V, k, p(ids), p(lp), None)
+    assert call(2, 64, 64, 800, 4, h=None) == binding.ERR_NULL
+    assert call(0, 64, 64, 800, 4) == binding.ERR_DIM
+    assert call(2, 64, 64, 800, 0) == binding.ERR_DIM
+    assert call(2, 64, 64, 800, 801) == binding.ERR_DIM
+    assert call(2, 64, 64, 800, 65) == binding.ERR_DIM
+    assert call(513, 64, 64, 800, 4) == binding.ERR_DIM
+    assert call(2, 64, 64, 200000, 4) == binding.ERR_DIM
+    assert ctx.launch_count() == n0
