@@ -181,7 +181,7 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         CK(stream_head(c->s.z, Bm, mrows, p.mt, K, V, k, mode,
                        mode == 0 ? ids + (size_t)m0 * k : nullptr,
                        mode == 0 ? logprobs + (size_t)m0 * k : nullptr,
-                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, true, st));
+                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, getenv("SLIMSPEC_DEBUG_NOPDL") == nullptr, st));
         c->launches += 2;
     }
     return SLIMSPEC_OK;

@@ -12,7 +12,6 @@ namespace slimspec {
 
 static constexpr int kRowsPerStage = 16;     // rows of the K x V matrix per pipeline stage
 static constexpr int kColThreads = 128;      // threads across one pass's columns, 8 columns each
-static constexpr int kMaxPassCols = kColThreads * 8;
 static constexpr int kEpiWarps = 4;
 static constexpr int kMaxStages = 12;
 static constexpr int kMaxCtas = 256;         // slabs per row the merge can take (8 lists per lane)
@@ -310,6 +309,7 @@ __global__ void __launch_bounds__(32 + 128 * KG + 32 * kEpiWarps, 1) k_stream_he
             if (pass > 0 && !mbar_wait(acc_free, (pass - 1) & 1, abort_flag, p.err, ERR_WAIT_FREE)) { alive = false; break; }
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
+                if (!active) break;        // columns past the pass would land in the next group's row
                 float* dst = part_s + ((size_t)g * MT + m) * pass_cols + ct * 8;
                 *reinterpret_cast<float4*>(dst) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
                 *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
@@ -530,9 +530,11 @@ static bool geometry(int mt, int K, int V, int k, int sm_count, Geometry* g)
     int ns = (int)(((size_t)kSmemBudget - fixed) / stage);
     if (ns > kMaxStages) ns = kMaxStages;
     g->nstages = ns;
-    g->smem = fixed + (size_t)ns * stage;
-    // the last CTA's merge keeps 2*P*k words per epilogue warp in the stage area
-    if ((size_t)kEpiWarps * 2 * ncta * k * 4 > (size_t)ns * stage) return false;
+    // the last CTA's merge keeps 2*P*k words per epilogue warp in the (then idle) stage area
+    const size_t merge = (size_t)kEpiWarps * 2 * ncta * k * 4;
+    if (fixed + merge > (size_t)kSmemBudget) return false;
+    const size_t area = (size_t)ns * stage > merge ? (size_t)ns * stage : merge;
+    g->smem = fixed + area;
     return true;
 }
 
