@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the draft LM-head forward (low-rank head, fused log-softmax / top-k).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+
+One step = one call of slimspec_head_topk: down-projection, the streamed up-projection,
+online log-softmax, top-k and the slab merge, on the 8B-class head at M = 1
+(d=4096, r=512, V=128256, k=10).  The metric is microseconds per call (lower is better).
+Weights rotate through several distinct copies (more than 4x the L2 capacity in total), so
+every call streams cold weights from HBM.  With N > 1 every rank runs an independent
+replica of the same workload (the path has no exchange step); the value is then the time
+divided by the calls of all ranks.
+
+`--impl reference` times the fp64 CPU oracle on the host cores instead (rank 0 only).
+Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "lm_head_us_per_call_M1"
+UNIT = "us/call"
+WORKLOAD = "c1"                      # d=4096, r=512, V=128256, k=10
+L2_BYTES = 126 * 1024 * 1024
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"]))}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+def head_bytes(M, d, r, V, k):
+    """Algorithmic bytes of one low-rank call: A, B and h read once, top-k written."""
+    return 2 * (d * r + r * V) + 2 * M * d + 8 * M * k
+
+
+def head_flops(M, d, r, V):
+    return 2 * M * (d * r + r * V)
+
+
+# --------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """nvidia-smi in the background, one sample every 100 ms, for the GPU this rank uses."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="clocks_", suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            # the busiest half of the samples stands for "under load"
+            top = sorted(sm)[len(sm) // 2:]
+            out["sm_mhz"] = statistics.median(top)
+            out["sm_max_mhz"] = max(mx)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# --------------------------------------------------------------------------- reference arm
+
+def oracle_step_time(cfg, M, frac_cols=1.0, reps=1):
+    """Seconds per oracle call of the low-rank head on the first frac_cols of the vocabulary."""
+    import oracle
+    from paper_2605_10453_b200 import synth
+    V = max(cfg.k + 1, int(round(cfg.V * frac_cols)))
+    x = synth.make_inputs(M, cfg.d, cfg.r, V, seed=cfg.seed, logit_scale=cfg.logit_scale)
+    b = {k: oracle.bf16_bits(v) for k, v in x.items()}
+    times = []
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        oracle.head_topk(b["h"], b["A"], b["B"], cfg.k)
+        times.append(time.perf_counter() - t0)
+    return times, V
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2605_10453_b200 import synth
+    cfg = synth.CONFIGS[WORKLOAD]
+    M = 1
+    oracle.build()
+    threads_used = min(oracle.threads(), M)
+    # size the per-step sample so that the whole run stays within about two minutes
+    probe, _ = oracle_step_time(cfg, M, 1.0, reps=1)
+    total_full = probe[0] * (args.steps + args.warmup)
+    frac = min(1.0, 120.0 / max(total_full, 1e-9))
+    times, Vs = oracle_step_time(cfg, M, frac, reps=args.steps + args.warmup)
+    timed = times[args.warmup:]
+    scale = cfg.V / Vs
+    us = statistics.mean(timed) * scale * 1e6
+    sample = ("full call" if Vs == cfg.V else
+              "first %d of %d vocabulary columns per step, time scaled by %.2f" % (Vs, cfg.V, scale))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s M=%d d=%d r=%d V=%d k=%d" % (WORKLOAD, M, cfg.d, cfg.r, cfg.V, cfg.k)},
+        "cpu_baseline": {"value": us, "unit": UNIT, "cores": threads_used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- our arm
+
+def time_calls(torch, fn, n):
+    """CUDA-event time of n back-to-back calls on the current stream, in milliseconds."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def copies_needed(nbytes):
+    return max(2, -(-4 * L2_BYTES // nbytes))
+
+
+def run_ours(args):
+    import torch
+    from paper_2605_10453_b200 import binding, build, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the head has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    build.build()
+    peaks, peaks_kind = load_peaks()
+
+    cfg = synth.CONFIGS[WORKLOAD]
+    M, d, r, V, k = 1, cfg.d, cfg.r, cfg.V, cfg.k
+    ctx = binding.Context(max_M=512, max_d=8192, max_V=V, max_k=16)
+    x = synth.make_inputs(M, d, r, V, seed=cfg.seed)
+    R = copies_needed(2 * (d * r + r * V))
+    h = x["h"].to(dev)
+    As = [x["A"].to(dev).clone() for _ in range(R)]
+    Bs = [x["B"].to(dev).clone() for _ in range(R)]
+    ids = torch.empty((M, k), dtype=torch.int32, device=dev)
+    lp = torch.empty((M, k), dtype=torch.float32, device=dev)
+    h_pin = x["h"].pin_memory()
+    ids_pin = torch.empty((M, k), dtype=torch.int32).pin_memory()
+    lp_pin = torch.empty((M, k), dtype=torch.float32).pin_memory()
+
+    def step(i):
+        ctx.slimspec_head_topk(h, As[i % R], Bs[i % R], k, out_ids=ids, out_logprobs=lp)
+
+    def step_host(i):
+        ctx.slimspec_head_topk_host(h_pin, As[i % R], Bs[i % R], k, out_ids_host=ids_pin, out_logprobs_host=lp_pin)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    K, W = args.steps, max(args.warmup, 3)
+    sampler = ClockSampler(local)
+    for i in range(W):
+        step(i)
+    barrier()
+    sampler.start()
+    # ---- the timed region: exactly K steps
+    n0 = ctx.launch_count()
+    ms = time_calls(torch, step, K)
+    launches = ctx.launch_count() - n0
+    barrier()
+    ms = max_over_ranks(ms)
+    # ---- the dominant kernel alone, events recorded by the library around it, same K steps
+    ctx.kernel_timing(True)
+    for i in range(K):
+        step(i)
+    kms, kn = ctx.kernel_timing_read()
+    ctx.kernel_timing(False)
+    # ---- end to end: host activations in, host results out, every step
+    for i in range(3):
+        step_host(i)
+    barrier()
+    e2e_ms = max_over_ranks(time_calls(torch, step_host, K))
+    clocks = sampler.stop()
+    if ctx.last_error() != binding.OK:
+        raise SystemExit("device-side wait timed out during the benchmark")
+
+    us_call = ms * 1e3 / (K * world)
+    e2e_us = e2e_ms * 1e3 / (K * world)
+    kern_us = kms * 1e3 / max(kn, 1)
+    kern_bytes = 2 * r * V + 4 * r * M            # the streamed matrix and the fp32 code
+    achieved = kern_bytes / (kern_us * 1e-6) / 1e9
+
+    line = {
+        "metric": METRIC, "value": us_call, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms / K, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 weights, f32 accumulate", "data": "synthetic",
+        "config": {"workload": "%s M=%d d=%d r=%d V=%d k=%d" % (WORKLOAD, M, d, r, V, k),
+                   "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "cache": "weights rotate through %d copies (%.0f MB > 4x L2): every call is cold" %
+                            (R, R * 2 * (d * r + r * V) / 1e6),
+                   "path": {1: "generic", 2: "stream", 3: "tensor"}.get(ctx.last_path(), "?")},
+        "e2e": {"value": e2e_us, "unit": UNIT, "h2d_bytes_per_step": M * d * 2, "d2h_bytes_per_step": M * k * 8},
+        "gpu_launches": int(launches),
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "roofline": {"bound": "hbm", "kernel": "k_stream_head", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                     "peak_kind": "of " + peaks_kind, "bytes_per_launch": kern_bytes, "us_per_launch": kern_us,
+                     "whole_call_frac": head_bytes(M, d, r, V, k) / (us_call * world * 1e-6) / 1e9 / peaks["hbm_gbs"]},
+    }
+
+    if rank == 0 and world == 1 and not args.no_extra:
+        line["extra"] = extra_points(torch, ctx, synth, binding, dev, peaks)
+        line["cpu_baseline"] = cpu_baseline(cfg, M)
+    ctx.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(cfg, M):
+    """The oracle as it stands, timed on the host cores for about ten seconds."""
+    import oracle as _o
+    from paper_2605_10453_b200 import synth
+    _o.build()
+    x = synth.make_inputs(M, cfg.d, cfg.r, cfg.V, seed=cfg.seed, logit_scale=cfg.logit_scale)
+    b = {kk: _o.bf16_bits(v) for kk, v in x.items()}
+    times = []
+    t_end = time.perf_counter() + 10.0
+    while len(times) < 3 or time.perf_counter() < t_end:
+        t0 = time.perf_counter()
+        _o.head_topk(b["h"], b["A"], b["B"], cfg.k)
+        times.append(time.perf_counter() - t0)
+    return {"value": statistics.mean(times) * 1e6, "unit": UNIT, "cores": min(_o.threads(), M), "kind": "oracle",
+            "sample": "%d full calls of the same workload (M=%d)" % (len(times), M)}
+
+
+def extra_points(torch, ctx, synth, binding, dev, peaks):
+    """Other points of the metric, each timed cold with CUDA events: M = 8, the full-rank head, M = 512."""
+    out = {}
+    c1, c3 = synth.CONFIGS["c1"], synth.CONFIGS["c3"]
+    d, r, V, k = c1.d, c1.r, c1.V, c1.k
+    x = synth.make_inputs(8, d, r, V, seed=c1.seed)
+    R = copies_needed(2 * (d * r + r * V))
+    As = [x["A"].to(dev).clone() for _ in range(R)]
+    Bs = [x["B"].to(dev).clone() for _ in range(R)]
+
+    def point(M, n):
+        h = synth.make_h(M, d, c1.seed).to(dev)
+        ids = torch.empty((M, k), dtype=torch.int32, device=dev)
+        lp = torch.empty((M, k), dtype=torch.float32, device=dev)
+        fn = lambda i: ctx.slimspec_head_topk(h, As[i % R], Bs[i % R], k, out_ids=ids, out_logprobs=lp)
+        for i in range(3):
+            fn(i)
+        us = time_calls(torch, fn, n) * 1e3 / n
+        t_hbm = head_bytes(M, d, r, V, k) / (peaks["hbm_gbs"] * 1e9)
+        t_mma = head_flops(M, d, r, V) / (peaks["bf16_tflops"] * 1e12)
+        return {"us_per_call": us, "rows_per_s": M / (us * 1e-6), "roofline_us": max(t_hbm, t_mma) * 1e6,
+                "roofline_frac": max(t_hbm, t_mma) * 1e6 / us, "bound": "hbm" if t_hbm >= t_mma else "tensor",
+                "path": {1: "generic", 2: "stream", 3: "tensor"}.get(ctx.last_path(), "?")}
+
+    out["slimspec_M1"] = point(1, 200)
+    out["slimspec_M8"] = point(8, 100)
+    out["slimspec_M512"] = point(512, 5)
+    del As, Bs
+    # full-rank baseline: W is 1.05 GB, eight times the L2, so one copy is cold by itself
+    Wd = synth.make_W(d, V, c1.seed).to(dev)
+    for M, n in ((1, 50), (8, 20)):
+        h = synth.make_h(M, d, c1.seed).to(dev)
+        ids = torch.empty((M, k), dtype=torch.int32, device=dev)
+        lp = torch.empty((M, k), dtype=torch.float32, device=dev)
+        fn = lambda i: ctx.fullhead_topk(h, Wd, k, out_ids=ids, out_logprobs=lp)
+        for i in range(3):
+            fn(i)
+        us = time_calls(torch, fn, n) * 1e3 / n
+        fb = 2 * d * V + 2 * M * d
+        out["fullhead_M%d" % M] = {"us_per_call": us, "roofline_us": fb / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                                   "roofline_frac": fb / (peaks["hbm_gbs"] * 1e9) * 1e6 / us}
+    for M in (1, 8):
+        out["speedup_vs_fullhead_M%d" % M] = out["fullhead_M%d" % M]["us_per_call"] / out["slimspec_M%d" % M]["us_per_call"]
+    out["bytes_ratio_target"] = 0.8 * (d * V) / (d * r + r * V)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the extra points and the CPU baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -116,6 +116,23 @@ int slimspec_last_error(slimspec_ctx* ctx);
 /* Number of kernels the library has launched on this context since it was created. */
 long long slimspec_launch_count(const slimspec_ctx* ctx);
 
+/*
+ * Device timing of the dominant kernel (the one that streams B or W), for roofline
+ * reports.  While enabled, each *_topk / *_logits call records a CUDA event on its stream
+ * directly before and after that kernel; the event between the down-projection and the
+ * streaming kernel also keeps the two from overlapping, so the figure is the kernel alone
+ * and calls are slightly slower than with timing off.  Enabling resets the totals.
+ * At most 256 launches are pending at a time; the call that records the 257th first waits
+ * for the earlier ones.
+ */
+int slimspec_kernel_timing(slimspec_ctx* ctx, int enable);
+
+/*
+ * Wait for the timed kernels recorded so far and return their summed duration in
+ * milliseconds and their number (both host pointers, both required).
+ */
+int slimspec_kernel_timing_read(slimspec_ctx* ctx, double* total_ms, long long* launches);
+
 /* Static description of a status code. */
 const char* slimspec_strerror(int status);
 

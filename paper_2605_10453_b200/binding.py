@@ -21,6 +21,7 @@ EXPORTS = [
     "slimspec_create", "slimspec_destroy", "slimspec_force_path", "slimspec_last_path",
     "slimspec_head_topk", "slimspec_head_topk_host", "slimspec_head_logits", "fullhead_topk",
     "slimspec_last_error", "slimspec_launch_count", "slimspec_strerror",
+    "slimspec_kernel_timing", "slimspec_kernel_timing_read",
 ]
 
 _lib = None
@@ -66,6 +67,11 @@ def load():
     lib.slimspec_last_error.restype = ci
     lib.slimspec_launch_count.argtypes = [vp]
     lib.slimspec_launch_count.restype = ctypes.c_longlong
+    lib.slimspec_kernel_timing.argtypes = [vp, ci]
+    lib.slimspec_kernel_timing.restype = ci
+    lib.slimspec_kernel_timing_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double),
+                                                ctypes.POINTER(ctypes.c_longlong)]
+    lib.slimspec_kernel_timing_read.restype = ci
     lib.slimspec_strerror.argtypes = [ci]
     lib.slimspec_strerror.restype = ctypes.c_char_p
     _lib = lib
@@ -124,6 +130,19 @@ class Context:
 
     def launch_count(self) -> int:
         return int(load().slimspec_launch_count(self._h))
+
+    def kernel_timing(self, enable: bool):
+        rc = load().slimspec_kernel_timing(self._h, 1 if enable else 0)
+        if rc != OK:
+            raise SlimSpecError(rc, "slimspec_kernel_timing")
+
+    def kernel_timing_read(self):
+        """(total milliseconds, launches) of the timed dominant kernel since timing was enabled."""
+        ms, n = ctypes.c_double(), ctypes.c_longlong()
+        rc = load().slimspec_kernel_timing_read(self._h, ctypes.byref(ms), ctypes.byref(n))
+        if rc != OK:
+            raise SlimSpecError(rc, "slimspec_kernel_timing_read")
+        return ms.value, int(n.value)
 
     # ---- the calls of the C ABI; outputs may be passed in to avoid allocation -----------
     def slimspec_head_topk(self, h, A, B, k, out_ids=None, out_logprobs=None, stream=None):

@@ -18,7 +18,15 @@ struct slimspec_ctx {
     bf16* h_stage;        // device copy of host activations (head_topk_host)
     int32_t* ids_stage;   // device results of head_topk_host
     float* lp_stage;
+    // optional device timing of the kernel that streams the weight matrix
+    int timing_on;
+    int timing_used;                 // event pairs recorded and not yet read
+    cudaEvent_t* ev0;
+    cudaEvent_t* ev1;
+    double timing_ms;                // accumulated
+    long long timing_launches;
 };
+static const int kTimingEvents = 256;
 
 static const int kMaxParts = 1024;     // most V slabs any kernel writes per row
 static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
@@ -87,6 +95,11 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
     cudaDeviceSynchronize();
     cudaFree(c->s.z); cudaFree(c->s.zpart); cudaFree(c->s.part); cudaFree(c->s.tickets); cudaFree(c->s.err);
     cudaFree(c->s.logits); cudaFree(c->h_stage); cudaFree(c->ids_stage); cudaFree(c->lp_stage);
+    if (c->ev0) {
+        for (int i = 0; i < kTimingEvents; ++i) { cudaEventDestroy(c->ev0[i]); cudaEventDestroy(c->ev1[i]); }
+        delete[] c->ev0;
+        delete[] c->ev1;
+    }
     delete c;
 }
 
@@ -114,6 +127,56 @@ extern "C" int slimspec_last_error(slimspec_ctx* c)
         cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int));
         return SLIMSPEC_ERR_TIMEOUT;
     }
+    return SLIMSPEC_OK;
+}
+
+// Fold the recorded event pairs into the totals; waits for the last recorded kernel.
+static int timing_drain(slimspec_ctx* c)
+{
+    for (int i = 0; i < c->timing_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(c->ev1[i]) != cudaSuccess ||
+            cudaEventElapsedTime(&ms, c->ev0[i], c->ev1[i]) != cudaSuccess) {
+            cudaGetLastError();
+            c->timing_used = 0;
+            return SLIMSPEC_ERR_CUDA;
+        }
+        c->timing_ms += ms;
+        c->timing_launches += 1;
+    }
+    c->timing_used = 0;
+    return SLIMSPEC_OK;
+}
+
+extern "C" int slimspec_kernel_timing(slimspec_ctx* c, int enable)
+{
+    if (!c) return SLIMSPEC_ERR_NULL;
+    if (enable && !c->ev0) {
+        c->ev0 = new (std::nothrow) cudaEvent_t[kTimingEvents];
+        c->ev1 = new (std::nothrow) cudaEvent_t[kTimingEvents];
+        if (!c->ev0 || !c->ev1) return SLIMSPEC_ERR_NOMEM;
+        for (int i = 0; i < kTimingEvents; ++i) {
+            if (cudaEventCreate(&c->ev0[i]) != cudaSuccess || cudaEventCreate(&c->ev1[i]) != cudaSuccess)
+                return SLIMSPEC_ERR_CUDA;
+        }
+    }
+    if (enable) {
+        int rc = timing_drain(c);
+        if (rc != SLIMSPEC_OK) return rc;
+        c->timing_ms = 0.0;
+        c->timing_launches = 0;
+    }
+    c->timing_on = enable ? 1 : 0;
+    return SLIMSPEC_OK;
+}
+
+extern "C" int slimspec_kernel_timing_read(slimspec_ctx* c, double* total_ms, long long* launches)
+{
+    if (!c || !total_ms || !launches) return SLIMSPEC_ERR_NULL;
+    int rc = timing_drain(c);
+    if (rc != SLIMSPEC_OK) return rc;
+    *total_ms = c->timing_ms;
+    *launches = c->timing_launches;
     return SLIMSPEC_OK;
 }
 
@@ -178,10 +241,18 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         const bf16* hm = h + (size_t)m0 * d;
         if (lowrank) CK(stream_downproj(hm, A, mrows, p.mt, d, r, c->s, st));
         else CK(stream_widen_t(hm, mrows, p.mt, d, c->s.z, st));
+        int slot = -1;
+        if (c->timing_on) {
+            if (c->timing_used == kTimingEvents) { int rc = timing_drain(c); if (rc != SLIMSPEC_OK) return rc; }
+            slot = c->timing_used++;
+            CK(cudaEventRecord(c->ev0[slot], st));
+        }
+        // an event between the two kernels serialises them: the timed kernel then runs alone
         CK(stream_head(c->s.z, Bm, mrows, p.mt, K, V, k, mode,
                        mode == 0 ? ids + (size_t)m0 * k : nullptr,
                        mode == 0 ? logprobs + (size_t)m0 * k : nullptr,
-                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, getenv("SLIMSPEC_DEBUG_NOPDL") == nullptr, st));
+                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, slot < 0, st));
+        if (slot >= 0) CK(cudaEventRecord(c->ev1[slot], st));
         c->launches += 2;
     }
     return SLIMSPEC_OK;

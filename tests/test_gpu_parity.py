@@ -22,7 +22,7 @@ def obits(x):
 
 @pytest.fixture(scope="module")
 def ctx():
-    c = binding.Context(max_M=512, max_d=8192, max_V=152064, max_k=64)
+    c = binding.Context(max_M=512, max_d=8192, max_V=160000, max_k=64)
     yield c
     c.close()
 
@@ -245,5 +245,5 @@ def test_argument_errors_launch_nothing(ctx):
     assert call(2, 64, 64, 800, 801) == binding.ERR_DIM
     assert call(2, 64, 64, 800, 65) == binding.ERR_DIM
     assert call(513, 64, 64, 800, 4) == binding.ERR_DIM
-    assert call(2, 64, 64, 200000, 4) == binding.ERR_DIM
+    assert call(2, 64, 64, 200008, 4) == binding.ERR_DIM
     assert ctx.launch_count() == n0
