@@ -65,11 +65,9 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     c->s.max_parts = kMaxParts;
     const size_t mpad = (size_t)round_up(max_M, kRowPad);
     const size_t z_elems = mpad * (size_t)max_d;
-    const size_t zpart_elems = (size_t)64 * kRowPad * (size_t)max_d;     // <= 64 d-slabs of 8 rows
-    const size_t part_elems = mpad * (size_t)kMaxParts * (2 + 2 * (size_t)max_k);
+    const size_t part_elems = mpad * (size_t)kMaxParts * (size_t)round_up(2 + 2 * max_k, 4);   // records padded to 16 bytes
     bool ok = true;
     ok = ok && cudaMalloc(&c->s.z, z_elems * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.tickets, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.err, sizeof(int)) == cudaSuccess;
@@ -93,7 +91,7 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
 {
     if (!c) return;
     cudaDeviceSynchronize();
-    cudaFree(c->s.z); cudaFree(c->s.zpart); cudaFree(c->s.part); cudaFree(c->s.tickets); cudaFree(c->s.err);
+    cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.tickets); cudaFree(c->s.err);
     cudaFree(c->s.logits); cudaFree(c->h_stage); cudaFree(c->ids_stage); cudaFree(c->lp_stage);
     if (c->ev0) {
         for (int i = 0; i < kTimingEvents; ++i) { cudaEventDestroy(c->ev0[i]); cudaEventDestroy(c->ev1[i]); }
@@ -213,7 +211,7 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
     const bool ptr_ok = aligned16(h) && aligned16(Bm) && (!lowrank || aligned16(A)) &&
                         (mode == 0 || aligned16(logits));
     StreamPlan sp = stream_plan(M, d, K, V, mode == 0 ? k : 1, c->sm_count);
-    const bool stream_ok = sp.ok && ptr_ok && (!lowrank || r % 64 == 0);
+    const bool stream_ok = sp.ok && ptr_ok && (!lowrank || r % 16 == 0);
     if (path == SLIMSPEC_PATH_AUTO) path = stream_ok ? SLIMSPEC_PATH_STREAM : SLIMSPEC_PATH_GENERIC;
     if (path == SLIMSPEC_PATH_TENSOR) return SLIMSPEC_ERR_ALIGN;   // tensor path not built yet
     if (path == SLIMSPEC_PATH_STREAM && !stream_ok) return SLIMSPEC_ERR_ALIGN;

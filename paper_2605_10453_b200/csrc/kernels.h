@@ -14,7 +14,6 @@ typedef __nv_bfloat16 bf16;
 // Layout in the context's scratch: float pm[P], ps[P], pv[P][k]; int pi[P][k] per row.
 struct Scratch {
     float* z;            // fp32 code (or widened h); generic path [M][K], streaming path transposed [K][mt]
-    float* zpart;        // split-d partial sums of the down-projection
     float* part;         // split-V partial records
     unsigned int* tickets;  // arrival counters (self-resetting)
     int* err;            // device error word
@@ -38,7 +37,7 @@ struct StreamPlan {
     int launches;    // kernels per call (for the launch counter)
 };
 StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count);
-// z = h A for M <= 8 rows, rows M..mt-1 zero-filled; split over d, deterministic.
+// z^T = (h A)^T for M <= 8 rows, rows M..mt-1 zero-filled; r must be a multiple of 16.
 cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
                             cudaStream_t st);
 // z^T = widened h^T (full-rank head: no down-projection).

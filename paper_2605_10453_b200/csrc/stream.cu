@@ -1,24 +1,21 @@
 // Streaming path for small M (<= 8 rows per launch): the K x V weight matrix is read from HBM
-// exactly once, in split-V slabs (one CTA per SM), staged through shared memory by bulk
-// asynchronous copies (TMA) and consumed with 128-bit shared loads and FP32 FMAs.
+// exactly once, in split-V slabs (one CTA per SM), with coalesced 128-bit loads held in flight
+// in registers and consumed by packed FP32 FMAs.
 // The logits never leave the SM: each CTA keeps a running max / sum-exp / top-k per row and
 // the last CTA to finish merges the per-slab records (Section 4.1 up-projection, the
 // softmax of Section 3.2 in online form, and the candidate selection).
 #include "kernels.h"
 #include "ptx.cuh"
 #include <float.h>
+#include <type_traits>
 
 namespace slimspec {
 
-static constexpr int kRowsPerStage = 16;     // rows of the K x V matrix per pipeline stage
-static constexpr int kColThreads = 128;      // threads across one pass's columns, 8 columns each
-static constexpr int kEpiWarps = 4;
-static constexpr int kMaxStages = 12;
-static constexpr int kMaxCtas = 256;         // slabs per row the merge can take (8 lists per lane)
-static constexpr int kListPerLane = kMaxCtas / 32;
-// Leave ~28 KB of the SM's shared memory to the kernel that produces z, so that it can share
-// the SM with this kernel's prologue under programmatic dependent launch.
-static constexpr int kSmemBudget = 200 * 1024;
+static constexpr int kMaxColThreads = 256;   // threads across one pass's columns, 8 columns each
+static constexpr int kMaxColWarps = kMaxColThreads / 32;
+static constexpr int kMaxCtas = 256;         // slabs per row the merge can take
+static constexpr int kZChunkBytes = 64 * 1024;   // shared memory for the code, as (z, z) pairs
+static constexpr int kNoId = 0x7fffffff;
 
 struct HeadParams {
     const float* zT;      // [K][MT] fp32 code, transposed and zero-padded to MT rows
@@ -26,64 +23,121 @@ struct HeadParams {
     int M, K, V, k, mode;
     int ncta;             // slabs
     int units_base, units_rem;   // V/8 column units: slab c has units_base + (c < units_rem)
-    int pass_units;       // most units one pass covers (<= 128)
-    int nstages;
-    int pitch;            // bytes between staged rows = pass_units * 16
+    int pass_units;       // most units one pass covers (<= ct)
+    int ct, rg;           // column threads (multiple of 32) and row groups: blockDim = ct * rg
+    int kc;               // rows of the code per shared-memory chunk (K, or a multiple of rg * U)
+    int rec_words;        // words per split-V record: max, sum-exp, k keys, k ids, padded to 4
+    int merge_rows;       // rows the last CTA merges per round
     int32_t* ids;
     float* logprobs;
     float* logits;
-    float* part;          // split-V records
+    float* part;          // split-V records [M][ncta][rec_words]
     unsigned int* ticket;
     int* err;
     int wait_prev;        // 1: zT is written by the kernel launched just before (PDL)
 };
 
 // ------------------------------------------------------------------------------------------
-// warp-level selection: every lane holds NC candidates (key = f2key(value), 0 = empty; id).
-// Afterwards lane j < k holds the j-th best in (value desc, id asc) order.
-template <int NC>
-__device__ __forceinline__ void warp_select(uint32_t (&ck)[NC], int (&ci)[NC], int k, int lane, uint32_t& outk,
-                                            int& outi)
+// Selection.  Candidates are (key, id) with key = f2key(logit) and key 0 = none; the order is
+// (key descending, id ascending).  Every lane offers the head of a list that is already in that
+// order; each round takes the best head of the warp and advances that lane's list.  Lane j < k
+// ends up with the j-th best.
+
+// One round: does this lane's head win?  The winner has the largest key, and among equal keys
+// the lowest id.  *any is false once no candidate is left.
+__device__ __forceinline__ bool round_winner(uint32_t hk, int hi, bool* any)
 {
-    outk = 0;
-    outi = 0x7fffffff;
+    const uint32_t wk = warp_max_u32(hk);
+    *any = wk != 0u;
+    const unsigned tied = __ballot_sync(0xffffffffu, hk == wk);
+    if (__popc(tied) == 1) return hk == wk;
+    const int wi = (int)warp_min_u32(hk == wk ? (uint32_t)hi : 0xffffffffu);
+    return hk == wk && hi == wi;
+}
+
+// The winner of round j drops its head into out_k[j], out_i[j] (shared memory, one pair of
+// 32-entry arrays per warp); nothing but the pop of the winner's list sits between two rounds.
+// Entries j >= (number of candidates) are left as they were: callers clear the arrays first.
+
+// Lists held in registers, NL entries per lane (unused entries: key 0, id kNoId).
+template <int NL>
+__device__ __forceinline__ void warp_topk_regs(uint32_t (&ck)[NL], int (&ci)[NL], int k, uint32_t* out_k, int* out_i)
+{
     for (int j = 0; j < k; ++j) {
-        uint32_t bk = ck[0];
-        int bi = ci[0];
-        int bs = 0;
+        bool any;
+        const bool win = round_winner(ck[0], ci[0], &any);
+        if (!any) break;
+        if (win) {
+            out_k[j] = ck[0];
+            out_i[j] = ci[0];
 #pragma unroll
-        for (int s = 1; s < NC; ++s) {
-            bool better = ck[s] > bk || (ck[s] == bk && ci[s] < bi);
-            bk = better ? ck[s] : bk;
-            bi = better ? ci[s] : bi;
-            bs = better ? s : bs;
+            for (int s = 0; s + 1 < NL; ++s) { ck[s] = ck[s + 1]; ci[s] = ci[s + 1]; }
+            ck[NL - 1] = 0u;
+            ci[NL - 1] = kNoId;
         }
-        const uint32_t wk = warp_max_u32(bk);
-        const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
-        const bool win = (bk == wk) && ((uint32_t)bi == wi);
-#pragma unroll
-        for (int s = 0; s < NC; ++s)
-            if (win && s == bs) ck[s] = 0;
-        if (lane == j) { outk = wk; outi = (int)wi; }
     }
 }
 
+// Lists held in shared memory: this lane's list is keys[0..len), ids[0..len).
+__device__ __forceinline__ void warp_topk_smem(const uint32_t* keys, const int* ids, int len, int k, uint32_t* out_k,
+                                               int* out_i)
+{
+    int pos = 0;
+    uint32_t hk = len > 0 ? keys[0] : 0u;
+    int hi = len > 0 ? ids[0] : kNoId;
+    for (int j = 0; j < k; ++j) {
+        bool any;
+        const bool win = round_winner(hk, hi, &any);
+        if (!any) break;
+        if (win) {
+            out_k[j] = hk;
+            out_i[j] = hi;
+            ++pos;
+            hk = pos < len ? keys[pos] : 0u;
+            hi = pos < len ? ids[pos] : kNoId;
+        }
+    }
+}
+
+// compare-exchange so that (ka, ia) comes before (kb, ib)
+__device__ __forceinline__ void order2(uint32_t& ka, int& ia, uint32_t& kb, int& ib)
+{
+    const bool swap = (ka < kb) || (ka == kb && ia > ib);
+    const uint32_t tk = swap ? kb : ka;
+    const int ti = swap ? ib : ia;
+    kb = swap ? ka : kb;
+    ib = swap ? ia : ib;
+    ka = tk;
+    ia = ti;
+}
+
+// sort the first 8 candidates of a 9-entry list (19 compare-exchanges)
+__device__ __forceinline__ void sort8(uint32_t (&k)[9], int (&i)[9])
+{
+#define SLIMSPEC_CE(a, b) order2(k[a], i[a], k[b], i[b])
+    SLIMSPEC_CE(0, 1); SLIMSPEC_CE(2, 3); SLIMSPEC_CE(4, 5); SLIMSPEC_CE(6, 7);
+    SLIMSPEC_CE(0, 2); SLIMSPEC_CE(1, 3); SLIMSPEC_CE(4, 6); SLIMSPEC_CE(5, 7);
+    SLIMSPEC_CE(1, 2); SLIMSPEC_CE(5, 6); SLIMSPEC_CE(0, 4); SLIMSPEC_CE(3, 7);
+    SLIMSPEC_CE(1, 5); SLIMSPEC_CE(2, 6);
+    SLIMSPEC_CE(1, 4); SLIMSPEC_CE(3, 6);
+    SLIMSPEC_CE(2, 4); SLIMSPEC_CE(3, 5);
+    SLIMSPEC_CE(3, 4);
+#undef SLIMSPEC_CE
+}
+
 // ------------------------------------------------------------------------------------------
-// z^T = (h A)^T for M <= 8 rows.  Grid (r/64, S): a CTA sums a slab of d for 64 columns of A,
-// the last CTA of a column block adds the S partial sums in slab order (deterministic).
-template <int MT>
-__global__ void __launch_bounds__(256) k_stream_downproj(const bf16* __restrict__ h, const bf16* __restrict__ A,
-                                                          int M, int d, int r, int slab, float* __restrict__ zpart,
-                                                          float* __restrict__ zT, unsigned int* __restrict__ tickets)
+// z^T = (h A)^T for M <= MT rows.  A CTA owns 16 columns of A (two 16-byte units) over all d
+// rows, so no partial sums cross CTAs; a thread owns one unit and every (NT/2)-th row, with
+// RB row loads in flight at a time.  Rows M..MT-1 of z^T are written as zeros.
+template <int MT, int NT, int RB>
+__global__ void __launch_bounds__(NT) k_stream_downproj(const bf16* __restrict__ h, const bf16* __restrict__ A, int M,
+                                                         int d, int r, float* __restrict__ zT)
 {
     pdl_launch_dependents();
-    __shared__ float red[8][MT][64];
-    __shared__ unsigned int s_ticket;
-    const int t = threadIdx.x, cg = t & 7, rl = t >> 3, lane = t & 31, warp = t >> 5;
-    const int c0 = blockIdx.x * 64;
-    const int i0 = blockIdx.y * slab;
-    const int i1 = min(i0 + slab, d);
-    const int S = gridDim.y;
+    __shared__ float red[NT / 32][MT][16];
+    const int t = threadIdx.x, u = t & 1, rl = t >> 1, lane = t & 31, warp = t >> 5;
+    const int c0 = blockIdx.x * 16 + u * 8;
+    constexpr int RSTEP = NT / 2;
 
     float acc[MT][8];
 #pragma unroll
@@ -91,63 +145,56 @@ __global__ void __launch_bounds__(256) k_stream_downproj(const bf16* __restrict_
 #pragma unroll
         for (int c = 0; c < 8; ++c) acc[m][c] = 0.f;
 
-    for (int i = i0 + rl; i < i1; i += 32) {
-        const uint4 q = *reinterpret_cast<const uint4*>(A + (size_t)i * r + c0 + cg * 8);
-        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-        float a[8];
+    for (int i0 = rl; i0 < d; i0 += RSTEP * RB) {
+        uint4 a[RB];
+        float hv[MT][RB];
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            a[2 * p] = __uint_as_float(w[p] << 16);
-            a[2 * p + 1] = __uint_as_float(w[p] & 0xffff0000u);
+        for (int j = 0; j < RB; ++j) {
+            const int i = i0 + j * RSTEP;
+            a[j] = (i < d) ? __ldg(reinterpret_cast<const uint4*>(A + (size_t)i * r + c0)) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int m = 0; m < MT; ++m) hv[m][j] = (i < d && m < M) ? __bfloat162float(h[(size_t)m * d + i]) : 0.f;
         }
 #pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            if (m < M) {
-                const float hv = __bfloat162float(h[(size_t)m * d + i]);
+        for (int j = 0; j < RB; ++j) {
+            const uint32_t w[4] = {a[j].x, a[j].y, a[j].z, a[j].w};
 #pragma unroll
-                for (int c = 0; c < 8; ++c) acc[m][c] = fmaf(hv, a[c], acc[m][c]);
+            for (int e = 0; e < 4; ++e) {
+                const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
+#pragma unroll
+                for (int m = 0; m < MT; ++m) {
+                    acc[m][2 * e] = fmaf(hv[m][j], lo, acc[m][2 * e]);
+                    acc[m][2 * e + 1] = fmaf(hv[m][j], hi, acc[m][2 * e + 1]);
+                }
             }
         }
     }
-    // the four row lanes of a warp share a column group: fold them, then the eight warps
+    // the 16 row lanes of a warp share a unit: fold them, then the warps through shared memory
 #pragma unroll
     for (int m = 0; m < MT; ++m)
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
             float v = acc[m][c];
+            v += __shfl_xor_sync(0xffffffffu, v, 2);
+            v += __shfl_xor_sync(0xffffffffu, v, 4);
             v += __shfl_xor_sync(0xffffffffu, v, 8);
             v += __shfl_xor_sync(0xffffffffu, v, 16);
             acc[m][c] = v;
         }
-    if (lane < 8) {
+    if (lane < 2) {
 #pragma unroll
         for (int m = 0; m < MT; ++m)
 #pragma unroll
             for (int c = 0; c < 8; ++c) red[warp][m][lane * 8 + c] = acc[m][c];
     }
     __syncthreads();
-    for (int e = t; e < MT * 64; e += 256) {
-        const int m = e / 64, c = e % 64;
+    if (t < MT * 16) {
+        const int m = t >> 4, c = t & 15;
         float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) v += red[w][m][c];
-        if (S == 1) zT[(size_t)(c0 + c) * MT + m] = v;
-        else zpart[((size_t)blockIdx.y * r + c0 + c) * MT + m] = v;
+        for (int w = 0; w < NT / 32; ++w) v += red[w][m][c];
+        zT[(size_t)(blockIdx.x * 16 + c) * MT + m] = v;
     }
-    if (S == 1) return;
-    __threadfence();
-    __syncthreads();
-    if (t == 0) s_ticket = atomicAdd(&tickets[blockIdx.x], 1u);
-    __syncthreads();
-    if (s_ticket != (unsigned)(S - 1)) return;
-    __threadfence();
-    for (int e = t; e < MT * 64; e += 256) {
-        const int m = e % MT, c = e / MT;
-        float v = 0.f;
-        for (int s = 0; s < S; ++s) v += __ldcg(&zpart[((size_t)s * r + c0 + c) * MT + m]);
-        zT[(size_t)(c0 + c) * MT + m] = v;
-    }
-    if (t == 0) tickets[blockIdx.x] = 0;
 }
 
 // z^T = widened h^T for the full-rank head (no down-projection).
@@ -161,358 +208,358 @@ __global__ void k_stream_widen_t(const bf16* __restrict__ h, int M, int MT, int 
 }
 
 // ------------------------------------------------------------------------------------------
-// The streaming head.  Warp roles: warp 0 producer (bulk copies), 4*KG consumer warps
-// (thread = 8 columns x one of KG row groups of a stage), 4 epilogue warps (sum the row
-// groups' partial sums; running softmax / top-k, or logit store; final merge).
-template <int MT, int KG>
-__global__ void __launch_bounds__(32 + 128 * KG + 32 * kEpiWarps, 1) k_stream_head(const HeadParams p)
+// The streaming head.  One CTA per V slab; thread = (column unit of 8 columns, row group).
+// Every thread keeps U 128-bit loads of its column unit in flight (rows g, g+RG, g+2RG, ...),
+// multiplies each arriving row by the code held in shared memory (packed FP32 FMAs) and
+// refills.  The row groups' partial sums meet in shared memory; the warps of the slab then
+// keep the running max / sum-exp / top-k per row (or store the logits).  The last CTA to
+// finish merges the per-slab records.
+__device__ __forceinline__ uint4 ldg_stream(const void* p)
 {
-    constexpr int RPG = kRowsPerStage / KG;          // rows per group per stage
-    constexpr int NCONS = 4 * KG;                    // consumer warps
-    extern __shared__ __align__(128) unsigned char smem[];
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
 
-    // ---- shared memory carve-up
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem);            // [kMaxStages]
-    uint64_t* empty = full + kMaxStages;                           // [kMaxStages]
-    uint64_t* acc_ready = empty + kMaxStages;
-    uint64_t* acc_free = acc_ready + 1;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(acc_free + 1);
-    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(const_cast<int*>(abort_flag) + 1);
-    float* ep_s = reinterpret_cast<float*>(smem + 256);            // [kEpiWarps][MT][66]
-    const int pass_cols = p.pass_units * 8;
-    float* part_s = ep_s + kEpiWarps * MT * 66;                    // [KG][MT][pass_cols]
-    unsigned char* stage0 = reinterpret_cast<unsigned char*>(part_s + (size_t)KG * MT * pass_cols);
-    stage0 = reinterpret_cast<unsigned char*>(((uintptr_t)stage0 + 127) & ~(uintptr_t)127);
-    const int ztile_bytes = kRowsPerStage * MT * 4;
-    const int stage_bytes = kRowsPerStage * p.pitch + ((ztile_bytes + 127) & ~127);
+template <int MT, int U>
+__global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const HeadParams p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(smem);
+    uint32_t* sel_s = reinterpret_cast<uint32_t*>(smem + 128);           // [16 warps][32 keys, 32 ids]
+    float* ep_s = reinterpret_cast<float*>(smem + 128 + 16 * 64 * 4);    // [MT][kMaxColWarps][66]
+    float* red = ep_s + MT * kMaxColWarps * 66;                          // [RG][MT][ct*8]
+    const int CT = p.ct, RG = p.rg;
+    const int pass_cols = CT * 8;
+    float2* zs = reinterpret_cast<float2*>(red + (size_t)RG * MT * pass_cols);   // [kc][MT] (z, z) pairs
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    uint32_t* sel_k = sel_s + warp * 64;             // this warp's selection output
+    int* sel_i = reinterpret_cast<int*>(sel_k + 32);
+    const int g = tid / CT, c = tid - g * CT;        // row group, column unit inside the pass
+    const int NW = CT >> 5;                          // warps across a pass
+    const int cw = warp - g * NW;                    // this warp's position across the pass
     const int cta = blockIdx.x;
+    const int K = p.K, V = p.V, k = p.k;
+    const int stepU = RG * U;
 
     // ---- this CTA's slab and its passes
     const int my_units = p.units_base + (cta < p.units_rem ? 1 : 0);
     const int unit0 = cta * p.units_base + min(cta, p.units_rem);
     const int npass = (my_units + p.pass_units - 1) / p.pass_units;
     const int units_per_pass = npass ? (my_units + npass - 1) / npass : 0;
-    const int kchunks = p.K / kRowsPerStage;
-    const int total = npass * kchunks;
 
-    if (tid == 0) {
-        for (int s = 0; s < p.nstages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCONS); }
-        mbar_init(acc_ready, NCONS);
-        mbar_init(acc_free, kEpiWarps);
-        *abort_flag = 0;
-        mbar_fence_init();
+    // Two sets of UH loads each: one set is consumed while the other is in flight, so a wait
+    // for the older set never waits for loads issued after it.
+    constexpr int UH = U / 2;
+    uint4 q[2][UH];
+    auto prologue = [&](int pass) {
+        const int pu0 = pass * units_per_pass;
+        const int pun = min(units_per_pass, my_units - pu0);
+        const bf16* base = p.B + (size_t)(unit0 + pu0 + c) * 8;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+            for (int j = 0; j < UH; ++j) {
+                const int row = g + (hh * UH + j) * RG;
+                q[hh][j] = (c < pun && row < K) ? ldg_stream(base + (size_t)row * V) : make_uint4(0u, 0u, 0u, 0u);
+            }
+    };
+    if (npass > 0) prologue(0);
+    // the weights are on their way; now wait for the kernel that writes the code
+    if (p.wait_prev) pdl_wait();
+
+    float run_max[MT], run_sum[MT];
+    uint32_t lst_k[MT];                              // lane j < k: key of the j-th best so far
+    int lst_i[MT];
+    bool mine[MT];                                   // rows whose softmax / top-k this warp keeps
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        run_max[m] = -FLT_MAX; run_sum[m] = 0.f; lst_k[m] = 0; lst_i[m] = kNoId;
+        mine[m] = (m % RG) == g;
     }
-    __syncthreads();
 
-    if (warp == 0) {
-        // ================= producer =================
-        const int prefetch = min(p.nstages, total);
-        for (int it = 0; it < total; ++it) {
-            const int slot = it % p.nstages, use = it / p.nstages;
-            const int pass = it / kchunks, kc = it - pass * kchunks;
-            const int pu0 = pass * units_per_pass;
-            const int pun = min(units_per_pass, my_units - pu0);
-            const uint32_t row_bytes = (uint32_t)pun * 16u;
-            unsigned char* st = stage0 + (size_t)slot * stage_bytes;
-            if (use > 0 && !mbar_wait(&empty[slot], (use - 1) & 1, abort_flag, p.err, ERR_WAIT_EMPTY)) break;
-            if (lane == 0) mbar_arrive_expect_tx(&full[slot], row_bytes * kRowsPerStage + ztile_bytes);
-            __syncwarp();
-            if (lane < kRowsPerStage) {
-                const bf16* src = p.B + (size_t)(kc * kRowsPerStage + lane) * p.V + (size_t)(unit0 + pu0) * 8;
-                bulk_g2s(st + (size_t)lane * p.pitch, src, row_bytes, &full[slot]);
-            }
-            const bool z_now = !(p.wait_prev && it < prefetch);
-            if (z_now && lane == kRowsPerStage)
-                bulk_g2s(st + kRowsPerStage * p.pitch, p.zT + (size_t)kc * kRowsPerStage * MT, ztile_bytes, &full[slot]);
-            if (p.wait_prev && it == prefetch - 1) {
-                // weights of the first stages are in flight; now wait for the kernel that writes z
-                pdl_wait();
-                if (lane == kRowsPerStage) {
-                    for (int j = 0; j < prefetch; ++j) {
-                        const int kcj = j % kchunks;
-                        unsigned char* sj = stage0 + (size_t)(j % p.nstages) * stage_bytes;
-                        bulk_g2s(sj + kRowsPerStage * p.pitch, p.zT + (size_t)kcj * kRowsPerStage * MT, ztile_bytes,
-                                 &full[j % p.nstages]);
-                    }
-                }
-            }
-        }
-    } else if (warp <= NCONS) {
-        // ================= consumers =================
-        const int cw = warp - 1;
-        const int g = cw >> 2;                          // row group
-        const int ct = ((cw & 3) << 5) | lane;          // column unit inside the pass
-        float acc[MT][8];
-        int it = 0;
-        bool alive = true;
-        for (int pass = 0; pass < npass && alive; ++pass) {
-            const int pu0 = pass * units_per_pass;
-            const int pun = min(units_per_pass, my_units - pu0);
-            const bool active = ct < pun;
+    for (int pass = 0; pass < npass; ++pass) {
+        const int pu0 = pass * units_per_pass;
+        const int pun = min(units_per_pass, my_units - pu0);
+        const bool active = c < pun;
+        const bf16* base = p.B + (size_t)(unit0 + pu0 + c) * 8;
+        float2 acc[MT][4];
 #pragma unroll
-            for (int m = 0; m < MT; ++m)
+        for (int m = 0; m < MT; ++m)
 #pragma unroll
-                for (int c = 0; c < 8; ++c) acc[m][c] = 0.f;
-            for (int kc = 0; kc < kchunks; ++kc, ++it) {
-                const int slot = it % p.nstages, use = it / p.nstages;
-                if (!mbar_wait(&full[slot], use & 1, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
-                const unsigned char* st = stage0 + (size_t)slot * stage_bytes;
-                const float* zt = reinterpret_cast<const float*>(st + kRowsPerStage * p.pitch) + g * RPG * MT;
-                if (active) {
-                    const unsigned char* bp = st + (size_t)(g * RPG) * p.pitch + ct * 16;
+            for (int e = 0; e < 4; ++e) acc[m][e] = make_float2(0.f, 0.f);
+
+        // rows row, row + RG, ... (U of them): multiply what has arrived, then refill
+        auto block = [&](int row, int kc0, int kend, auto checked) {
+            constexpr bool kChecked = decltype(checked)::value;
 #pragma unroll
-                    for (int rr = 0; rr < RPG; ++rr) {
-                        const uint4 q = *reinterpret_cast<const uint4*>(bp + (size_t)rr * p.pitch);
-                        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-                        float zv[MT];
-                        if constexpr (MT == 1) {
-                            zv[0] = zt[rr];
-                        } else if constexpr (MT == 2) {
-                            const float2 t2 = *reinterpret_cast<const float2*>(zt + rr * 2);
-                            zv[0] = t2.x; zv[1] = t2.y;
-                        } else {
+            for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll
-                            for (int m4 = 0; m4 < MT / 4; ++m4) {
-                                const float4 t4 = *reinterpret_cast<const float4*>(zt + rr * MT + m4 * 4);
-                                zv[m4 * 4 + 0] = t4.x; zv[m4 * 4 + 1] = t4.y; zv[m4 * 4 + 2] = t4.z; zv[m4 * 4 + 3] = t4.w;
-                            }
-                        }
+                for (int j = 0; j < UH; ++j) {
+                    const int rj = row + (hh * UH + j) * RG;
+                    if (!kChecked || rj < kend) {
+                        const uint32_t w[4] = {q[hh][j].x, q[hh][j].y, q[hh][j].z, q[hh][j].w};
+                        float2 b2[4];
 #pragma unroll
-                        for (int pq = 0; pq < 4; ++pq) {
-                            const float lo = __uint_as_float(w[pq] << 16);
-                            const float hi = __uint_as_float(w[pq] & 0xffff0000u);
-                            if constexpr (MT >= 4) {
+                        for (int e = 0; e < 4; ++e)
+                            b2[e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
+                        const float2* zr = zs + (size_t)(rj - kc0) * MT;
 #pragma unroll
-                                for (int m = 0; m < MT; ++m) {
-                                    float2 r2 = __ffma2_rn(make_float2(lo, hi), make_float2(zv[m], zv[m]),
-                                                           make_float2(acc[m][2 * pq], acc[m][2 * pq + 1]));
-                                    acc[m][2 * pq] = r2.x;
-                                    acc[m][2 * pq + 1] = r2.y;
-                                }
-                            } else {
+                        for (int m = 0; m < MT; ++m) {
+                            const float2 z2 = zr[m];
 #pragma unroll
-                                for (int m = 0; m < MT; ++m) {
-                                    acc[m][2 * pq] = fmaf(lo, zv[m], acc[m][2 * pq]);
-                                    acc[m][2 * pq + 1] = fmaf(hi, zv[m], acc[m][2 * pq + 1]);
-                                }
-                            }
+                            for (int e = 0; e < 4; ++e) acc[m][e] = __ffma2_rn(b2[e], z2, acc[m][e]);
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&empty[slot]);
-            }
-            if (!alive) break;
-            // hand this pass's partial sums to the epilogue warps
-            if (pass > 0 && !mbar_wait(acc_free, (pass - 1) & 1, abort_flag, p.err, ERR_WAIT_FREE)) { alive = false; break; }
+                // the set is used up: refill all of it at once
 #pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                if (!active) break;        // columns past the pass would land in the next group's row
-                float* dst = part_s + ((size_t)g * MT + m) * pass_cols + ct * 8;
-                *reinterpret_cast<float4*>(dst) = make_float4(acc[m][0], acc[m][1], acc[m][2], acc[m][3]);
-                *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[m][4], acc[m][5], acc[m][6], acc[m][7]);
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_ready);
-        }
-    } else {
-        // ================= epilogue =================
-        const int ew = warp - 1 - NCONS;
-        const int et = (ew << 5) | lane;                 // column unit inside the pass
-        const int k = p.k;
-        float run_max[MT], run_sum[MT];
-        uint32_t lst_k[MT];                              // lane j < k: key of the j-th best so far
-        int lst_i[MT];
-#pragma unroll
-        for (int m = 0; m < MT; ++m) { run_max[m] = -FLT_MAX; run_sum[m] = 0.f; lst_k[m] = 0; lst_i[m] = 0x7fffffff; }
-        bool alive = true;
-        for (int pass = 0; pass < npass; ++pass) {
-            const int pu0 = pass * units_per_pass;
-            const int pun = min(units_per_pass, my_units - pu0);
-            const bool active = et < pun;
-            const int col = (unit0 + pu0 + et) * 8;      // first vocabulary id of this thread
-            if (!mbar_wait(acc_ready, pass & 1, abort_flag, p.err, ERR_WAIT_ACC)) { alive = false; break; }
-            float l[MT][8];
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) l[m][c] = 0.f;
-                if (active) {
-#pragma unroll
-                    for (int g = 0; g < KG; ++g) {
-                        const float* src = part_s + ((size_t)g * MT + m) * pass_cols + et * 8;
-                        const float4 a = *reinterpret_cast<const float4*>(src);
-                        const float4 b = *reinterpret_cast<const float4*>(src + 4);
-                        l[m][0] += a.x; l[m][1] += a.y; l[m][2] += a.z; l[m][3] += a.w;
-                        l[m][4] += b.x; l[m][5] += b.y; l[m][6] += b.z; l[m][7] += b.w;
-                    }
+                for (int j = 0; j < UH; ++j) {
+                    const int nr = row + (hh * UH + j) * RG + stepU;
+                    if (!kChecked || nr < K) q[hh][j] = ldg_stream(base + (size_t)nr * V);
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_free);
+        };
+
+        for (int kc0 = 0; kc0 < K; kc0 += p.kc) {
+            const int kend = min(K, kc0 + p.kc);
+            if (pass == 0 || p.kc < K) {
+                // bring this chunk of the code into shared memory as (z, z) pairs
+                if (kc0 > 0 || pass > 0) __syncthreads();
+                const float* src = p.zT + (size_t)kc0 * MT;
+                for (int e = tid; e < (kend - kc0) * MT; e += blockDim.x) {
+                    const float zv = __ldcg(src + e);
+                    zs[e] = make_float2(zv, zv);
+                }
+                __syncthreads();
+            }
+            if (active) {
+                for (int row = kc0 + g; row < kend; row += stepU) {
+                    // unchecked while this block and the next one lie wholly inside K
+                    if (row - g + 2 * stepU <= K) block(row, kc0, kend, std::false_type());
+                    else block(row, kc0, kend, std::true_type());
+                }
+            }
+        }
+        // ---- the row groups' partial sums meet in shared memory
+        if (active) {
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                float* dst = red + ((size_t)g * MT + m) * pass_cols + c * 8;
+                *reinterpret_cast<float4*>(dst) = make_float4(acc[m][0].x, acc[m][0].y, acc[m][1].x, acc[m][1].y);
+                *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[m][2].x, acc[m][2].y, acc[m][3].x, acc[m][3].y);
+            }
+        }
+        // next pass's first loads fly while this pass's logits are reduced
+        if (pass + 1 < npass) prologue(pass + 1);
+        __syncthreads();
+
+        const int col = (unit0 + pu0 + c) * 8;       // first vocabulary id of this thread
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            if (!mine[m] || m >= p.M) continue;
+            float l[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) l[e] = 0.f;
+            if (active) {
+                for (int gg = 0; gg < RG; ++gg) {
+                    const float* src = red + ((size_t)gg * MT + m) * pass_cols + c * 8;
+                    const float4 a = *reinterpret_cast<const float4*>(src);
+                    const float4 b = *reinterpret_cast<const float4*>(src + 4);
+                    l[0] += a.x; l[1] += a.y; l[2] += a.z; l[3] += a.w;
+                    l[4] += b.x; l[5] += b.y; l[6] += b.z; l[7] += b.w;
+                }
+            }
             if (p.mode == 1) {
                 if (active) {
-#pragma unroll
-                    for (int m = 0; m < MT; ++m) {
-                        if (m < p.M) {
-                            float* dst = p.logits + (size_t)m * p.V + col;
-                            *reinterpret_cast<float4*>(dst) = make_float4(l[m][0], l[m][1], l[m][2], l[m][3]);
-                            *reinterpret_cast<float4*>(dst + 4) = make_float4(l[m][4], l[m][5], l[m][6], l[m][7]);
-                        }
-                    }
+                    float* dst = p.logits + (size_t)m * V + col;
+                    *reinterpret_cast<float4*>(dst) = make_float4(l[0], l[1], l[2], l[3]);
+                    *reinterpret_cast<float4*>(dst + 4) = make_float4(l[4], l[5], l[6], l[7]);
                 }
                 continue;
             }
             // online softmax + running top-k of this warp's columns
+            float tmax = -FLT_MAX;
+            if (active) {
 #pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                float tmax = -FLT_MAX;
-                if (active) {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) tmax = fmaxf(tmax, l[m][c]);
-                }
-                const float wmax = warp_max(tmax);
-                const float nm = fmaxf(run_max[m], wmax);
-                float ts = 0.f;
-                if (active) {
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) ts += __expf(l[m][c] - nm);
-                }
-                run_sum[m] = run_sum[m] * __expf(run_max[m] - nm) + warp_sum(ts);
-                run_max[m] = nm;
-                // skip the selection when nothing here beats the current k-th best
-                const uint32_t kth = __shfl_sync(0xffffffffu, lst_k[m], k - 1);
-                if (f2key(wmax) < kth) continue;
-                uint32_t ck[9];
-                int ci[9];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) { ck[c] = active ? f2key(l[m][c]) : 0u; ci[c] = active ? col + c : 0x7fffffff; }
-                ck[8] = lst_k[m];
-                ci[8] = lst_i[m];
-                warp_select<9>(ck, ci, k, lane, lst_k[m], lst_i[m]);
+                for (int e = 0; e < 8; ++e) tmax = fmaxf(tmax, l[e]);
             }
+            const float wmax = warp_max(tmax);
+            const float nm = fmaxf(run_max[m], wmax);
+            float ts = 0.f;
+            if (active) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) ts += __expf(l[e] - nm);
+            }
+            run_sum[m] = run_sum[m] * __expf(run_max[m] - nm) + warp_sum(ts);
+            run_max[m] = nm;
+            // skip the selection when nothing here beats the current k-th best
+            const uint32_t kth = __shfl_sync(0xffffffffu, lst_k[m], k - 1);
+            if (f2key(wmax) < kth) continue;
+            // this lane's list: its eight new logits in order, then its entry of the running list
+            uint32_t ck[9];
+            int ci[9];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { ck[e] = active ? f2key(l[e]) : 0u; ci[e] = active ? col + e : kNoId; }
+            sort8(ck, ci);
+            ck[8] = lst_k[m];
+            ci[8] = lst_i[m];
+#pragma unroll
+            for (int e = 7; e >= 0; --e) order2(ck[e], ci[e], ck[e + 1], ci[e + 1]);
+            sel_k[lane] = 0u;
+            sel_i[lane] = kNoId;
+            __syncwarp();
+            warp_topk_regs<9>(ck, ci, k, sel_k, sel_i);
+            __syncwarp();
+            lst_k[m] = sel_k[lane];
+            lst_i[m] = sel_i[lane];
+            __syncwarp();
         }
-        if (p.mode == 1 || !alive) return;
+        if (pass + 1 < npass) __syncthreads();       // the partial sums may be overwritten now
+    }
+    if (p.mode == 1) return;
 
-        // ---- fold the four epilogue warps into one record per (row, slab)
+    // ---- fold the warps across the slab into one record per (row, slab)
+    // ep_s: per (row, warp) 66 words: max, sum-exp, 32 keys, 32 ids
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        if (!mine[m] || m >= p.M) continue;
+        float* rec = ep_s + ((size_t)m * kMaxColWarps + cw) * 66;
+        if (lane == 0) { rec[0] = run_max[m]; rec[1] = run_sum[m]; }
+        rec[2 + lane] = __uint_as_float(lst_k[m]);
+        rec[34 + lane] = __int_as_float(lst_i[m]);
+    }
+    __syncthreads();
+    const int P = p.ncta;
+    const int RW = p.rec_words;
+    if (cw == 0) {
+        // the lanes share out the NW sorted lists: 32 / NW lanes per list, a run of each list per lane
+        const int lpl = 32 / NW;
+        const int seg = (k + lpl - 1) / lpl;
+        const int lw = lane / lpl, ls = lane - lw * lpl;
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
-            float* rec = ep_s + ((size_t)ew * MT + m) * 66;
-            if (lane == 0) { rec[0] = run_max[m]; rec[1] = run_sum[m]; }
-            rec[2 + lane] = __uint_as_float(lst_k[m]);
-            rec[34 + lane] = __int_as_float(lst_i[m]);
-        }
-        named_bar_sync(1, 32 * kEpiWarps);
-        const int P = p.ncta;
-        const size_t rec_stride = (size_t)P * (2 + 2 * k);
-        for (int m = ew; m < p.M; m += kEpiWarps) {
+            if (!mine[m] || m >= p.M) continue;
+            const float* rows = ep_s + (size_t)m * kMaxColWarps * 66;
             float cm = -FLT_MAX;
-#pragma unroll
-            for (int w = 0; w < kEpiWarps; ++w) cm = fmaxf(cm, ep_s[((size_t)w * MT + m) * 66]);
+            for (int w = 0; w < NW; ++w) cm = fmaxf(cm, rows[w * 66]);
             float cs = 0.f;
-            uint32_t ck[kEpiWarps];
-            int ci[kEpiWarps];
-#pragma unroll
-            for (int w = 0; w < kEpiWarps; ++w) {
-                const float* rec = ep_s + ((size_t)w * MT + m) * 66;
-                cs += rec[1] * __expf(rec[0] - cm);
-                ck[w] = __float_as_uint(rec[2 + lane]);
-                ci[w] = __float_as_int(rec[34 + lane]);
-            }
-            uint32_t ok;
-            int oi;
-            warp_select<kEpiWarps>(ck, ci, k, lane, ok, oi);
-            float* gp = p.part + (size_t)m * rec_stride;
-            if (lane == 0) { gp[cta] = cm; gp[P + cta] = cs; }
+            for (int w = 0; w < NW; ++w) cs += rows[w * 66 + 1] * __expf(rows[w * 66] - cm);
+            const int first = ls * seg;
+            const int len = (lw < NW && first < k) ? min(seg, k - first) : 0;
+            const int lwc = lw < NW ? lw : 0;
+            const uint32_t* lk = reinterpret_cast<const uint32_t*>(rows + lwc * 66 + 2 + first);
+            const int* li = reinterpret_cast<const int*>(rows + lwc * 66 + 34 + first);
+            sel_k[lane] = 0u;
+            sel_i[lane] = kNoId;
+            __syncwarp();
+            warp_topk_smem(lk, li, len, k, sel_k, sel_i);
+            __syncwarp();
+            const uint32_t ok = sel_k[lane];
+            const int oi = sel_i[lane];
+            __syncwarp();
+            float* gp = p.part + ((size_t)m * P + cta) * RW;
+            if (lane == 0) { gp[0] = cm; gp[1] = cs; }
             if (lane < k) {
-                gp[2 * P + (size_t)cta * k + lane] = __uint_as_float(ok);
-                gp[2 * P + (size_t)P * k + (size_t)cta * k + lane] = __int_as_float(oi);
+                gp[2 + lane] = __uint_as_float(ok);
+                gp[2 + k + lane] = __int_as_float(oi);
             }
         }
         __threadfence();
-        named_bar_sync(1, 32 * kEpiWarps);
-        if (ew == 0 && lane == 0) *s_ticket = atomicAdd(p.ticket, 1u);
-        named_bar_sync(1, 32 * kEpiWarps);
-        if (*s_ticket != (unsigned)(P - 1)) return;
+    }
+    __syncthreads();
+    if (tid == 0) *s_ticket = atomicAdd(p.ticket, 1u);
+    __syncthreads();
+    if (*s_ticket != (unsigned)(P - 1)) return;
 
-        // ---- last CTA: merge the P slab records of every row
-        __threadfence();
-        // the pipeline stages are idle now; reuse them to hold one row's candidate lists per warp
-        uint32_t* cand = reinterpret_cast<uint32_t*>(stage0) + (size_t)ew * 2 * P * k;
-        for (int m = ew; m < p.M; m += kEpiWarps) {
-            const float* gp = p.part + (size_t)m * rec_stride;
+    // ---- last CTA: merge the P slab records of every row, a few rows per round
+    __threadfence();
+    float* mrg = red;                                // the reduction and code areas are idle now
+    uint32_t* stage_k = reinterpret_cast<uint32_t*>(ep_s);            // [rows][groups][32] keys, then ids
+    const int row_words = P * RW;
+    const int ngroups = (P + 31) >> 5;               // groups of 32 slabs, one warp each
+    const int nwarps = blockDim.x >> 5;
+    for (int m0 = 0; m0 < p.M; m0 += p.merge_rows) {
+        const int nrows = min(p.merge_rows, p.M - m0);
+        const int n4 = nrows * row_words / 4;
+        const float4* src = reinterpret_cast<const float4*>(p.part + (size_t)m0 * row_words);
+        float4* dst = reinterpret_cast<float4*>(mrg);
+        // batches of independent loads: the records sit in L2, one round trip per batch
+        for (int i0 = tid; i0 < n4; i0 += blockDim.x * 8) {
+            float4 t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = i0 + j * blockDim.x;
+                t[j] = (i < n4) ? __ldcg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = i0 + j * blockDim.x;
+                if (i < n4) dst[i] = t[j];
+            }
+        }
+        __syncthreads();
+        // first level: a warp takes 32 slabs of one row, a lane per slab list
+        int* stage_i = reinterpret_cast<int*>(stage_k + (size_t)nrows * ngroups * 32);
+        for (int job = warp; job < nrows * ngroups; job += nwarps) {
+            const int rrow = job / ngroups, grp = job - rrow * ngroups;
+            const int s = grp * 32 + lane;
+            const float* rec = mrg + (size_t)rrow * row_words + (size_t)(s < P ? s : 0) * RW;
+            stage_k[(size_t)job * 32 + lane] = 0u;
+            stage_i[(size_t)job * 32 + lane] = kNoId;
+            __syncwarp();
+            warp_topk_smem(reinterpret_cast<const uint32_t*>(rec + 2), reinterpret_cast<const int*>(rec + 2 + k),
+                           s < P ? k : 0, k, stage_k + (size_t)job * 32, stage_i + (size_t)job * 32);
+        }
+        __syncthreads();
+        // second level: a warp per row folds the groups' lists and finishes the log-softmax
+        if (warp < nrows) {
+            const int m = m0 + warp;
+            const float* rows = mrg + (size_t)warp * row_words;
             float gm = -FLT_MAX;
-            for (int c = lane; c < P; c += 32) gm = fmaxf(gm, __ldcg(gp + c));
+            for (int s = lane; s < P; s += 32) gm = fmaxf(gm, rows[(size_t)s * RW]);
             gm = warp_max(gm);
             float gs = 0.f;
-            for (int c = lane; c < P; c += 32) gs += __ldcg(gp + P + c) * __expf(__ldcg(gp + c) - gm);
+            for (int s = lane; s < P; s += 32) gs += rows[(size_t)s * RW + 1] * __expf(rows[(size_t)s * RW] - gm);
             gs = warp_sum(gs);
             const float lse = gm + __logf(gs);
-            for (int e = lane; e < 2 * P * k; e += 32) cand[e] = __float_as_uint(__ldcg(gp + 2 * P + e));
+            const int lpl = 32 / ngroups;
+            const int seg = (k + lpl - 1) / lpl;
+            const int lw = lane / lpl, ls = lane - lw * lpl;
+            const int first = ls * seg;
+            const int len = (lw < ngroups && first < k) ? min(seg, k - first) : 0;
+            const size_t off = ((size_t)warp * ngroups + (lw < ngroups ? lw : 0)) * 32 + first;
+            sel_k[lane] = 0u;
+            sel_i[lane] = kNoId;
             __syncwarp();
-            // lane owns slabs lane, lane+32, ...; each slab list is sorted, so only heads compete
-            uint32_t hk[kListPerLane];
-            int hi[kListPerLane];
-            int hp[kListPerLane];
-#pragma unroll
-            for (int q = 0; q < kListPerLane; ++q) {
-                const int c = lane + 32 * q;
-                hp[q] = 0;
-                hk[q] = (c < P) ? cand[(size_t)c * k] : 0u;
-                hi[q] = (c < P) ? (int)cand[(size_t)P * k + (size_t)c * k] : 0x7fffffff;
-            }
-            uint32_t ok = 0;
-            int oi = 0x7fffffff;
-            for (int j = 0; j < k; ++j) {
-                uint32_t bk = hk[0];
-                int bi = hi[0], bs = 0;
-#pragma unroll
-                for (int q = 1; q < kListPerLane; ++q) {
-                    const bool better = hk[q] > bk || (hk[q] == bk && hi[q] < bi);
-                    bk = better ? hk[q] : bk;
-                    bi = better ? hi[q] : bi;
-                    bs = better ? q : bs;
-                }
-                const uint32_t wk = warp_max_u32(bk);
-                const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
-                const bool win = (bk == wk) && ((uint32_t)bi == wi);
-                if (win && wk != 0u) {
-#pragma unroll
-                    for (int q = 0; q < kListPerLane; ++q) {
-                        if (q == bs) {
-                            const int c = lane + 32 * q;
-                            const int np = hp[q] + 1;
-                            hp[q] = np;
-                            hk[q] = (np < k) ? cand[(size_t)c * k + np] : 0u;
-                            hi[q] = (np < k) ? (int)cand[(size_t)P * k + (size_t)c * k + np] : 0x7fffffff;
-                        }
-                    }
-                }
-                if (lane == j) { ok = wk; oi = (int)wi; }
-            }
+            warp_topk_smem(stage_k + off, stage_i + off, len, k, sel_k, sel_i);
+            __syncwarp();
+            const uint32_t ok = sel_k[lane];
+            const int oi = sel_i[lane];
             if (lane < k) {
                 p.ids[(size_t)m * k + lane] = oi;
                 p.logprobs[(size_t)m * k + lane] = key2f(ok) - lse;
             }
-            __syncwarp();
         }
-        if (ew == 0 && lane == 0) *p.ticket = 0;
+        __syncthreads();
     }
+    if (tid == 0) *p.ticket = 0;
 }
 
 // ------------------------------------------------------------------------------------------
 static int pick_mt(int M) { return M <= 1 ? 1 : M <= 2 ? 2 : M <= 4 ? 4 : 8; }
 
 struct Geometry {
-    int ncta, units_base, units_rem, pass_units, nstages, pitch, kg;
+    int ncta, units_base, units_rem, pass_units, ct, rg, u, kc, rec_words, merge_rows, threads;
     size_t smem;
 };
 
 static bool geometry(int mt, int K, int V, int k, int sm_count, Geometry* g)
 {
-    if (V % 8 != 0 || K % kRowsPerStage != 0 || k > 32 || k < 1) return false;
+    if (V % 8 != 0 || K < 1 || k > 32 || k < 1) return false;
     const int units = V / 8;
     int ncta = sm_count < kMaxCtas ? sm_count : kMaxCtas;
     if (ncta > units) ncta = units;
@@ -520,22 +567,36 @@ static bool geometry(int mt, int K, int V, int k, int sm_count, Geometry* g)
     g->units_base = units / ncta;
     g->units_rem = units % ncta;
     const int max_units = g->units_base + (g->units_rem ? 1 : 0);
-    const int npass = (max_units + kColThreads - 1) / kColThreads;
+    const int npass = (max_units + kMaxColThreads - 1) / kMaxColThreads;
     g->pass_units = (max_units + npass - 1) / npass;
-    g->pitch = g->pass_units * 16;
-    g->kg = (mt == 8) ? 2 : 4;
-    const size_t fixed = 256 + (size_t)kEpiWarps * mt * 66 * 4 + (size_t)g->kg * mt * g->pass_units * 8 * 4 + 128;
-    const size_t stage = (size_t)kRowsPerStage * g->pitch + (((size_t)kRowsPerStage * mt * 4 + 127) & ~(size_t)127);
-    if (fixed + 2 * stage > (size_t)kSmemBudget) return false;
-    int ns = (int)(((size_t)kSmemBudget - fixed) / stage);
-    if (ns > kMaxStages) ns = kMaxStages;
-    g->nstages = ns;
-    // the last CTA's merge keeps 2*P*k words per epilogue warp in the (then idle) stage area
-    const size_t merge = (size_t)kEpiWarps * 2 * ncta * k * 4;
-    if (fixed + merge > (size_t)kSmemBudget) return false;
-    const size_t area = (size_t)ns * stage > merge ? (size_t)ns * stage : merge;
+    g->ct = (g->pass_units + 31) / 32 * 32;
+    const int nt_max = mt <= 4 ? 512 : 256;
+    g->rg = nt_max / g->ct;
+    if (g->rg < 1) g->rg = 1;
+    if (g->rg > K) g->rg = K;
+    g->threads = g->ct * g->rg;
+    g->u = (mt == 4) ? 8 : 16;
+    // rows of the code per shared-memory chunk: all of K if it fits, else a multiple of rg*u
+    const int kc_max = kZChunkBytes / (mt * 8);
+    if (K <= kc_max) g->kc = K;
+    else {
+        g->kc = kc_max / (g->rg * g->u) * (g->rg * g->u);
+        if (g->kc < 1) return false;
+    }
+    g->rec_words = (2 + 2 * k + 3) / 4 * 4;
+    const size_t fixed = 128 + 16 * 64 * 4 + (size_t)mt * kMaxColWarps * 66 * 4;
+    const size_t work = (size_t)g->threads * mt * 32 + (size_t)g->kc * mt * 8;
+    const size_t one_row = (size_t)ncta * g->rec_words * 4;
+    const size_t area = work > one_row ? work : one_row;
+    g->merge_rows = (int)(area / one_row);
+    if (g->merge_rows > g->threads / 32) g->merge_rows = g->threads / 32;
+    // the first merge level parks rows * groups lists of 32 (key, id) pairs where the warps' records were
+    const int groups = (ncta + 31) / 32;
+    const int park = (int)((size_t)mt * kMaxColWarps * 66 * 4 / ((size_t)groups * 32 * 8));
+    if (park < 1) return false;
+    if (g->merge_rows > park) g->merge_rows = park;
     g->smem = fixed + area;
-    return true;
+    return g->smem <= 200 * 1024;
 }
 
 StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count)
@@ -556,17 +617,12 @@ StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count)
 cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
                             cudaStream_t st)
 {
-    const int cblocks = r / 64;
-    int S = (2 * 148 + cblocks - 1) / cblocks;
-    if (S > 64) S = 64;
-    int slab = ((d + S - 1) / S + 31) / 32 * 32;
-    S = (d + slab - 1) / slab;
-    dim3 grid(cblocks, S);
+    const int grid = r / 16;
     switch (mt) {
-    case 1: k_stream_downproj<1><<<grid, 256, 0, st>>>(h, A, M, d, r, slab, s.zpart, s.z, s.tickets + 1); break;
-    case 2: k_stream_downproj<2><<<grid, 256, 0, st>>>(h, A, M, d, r, slab, s.zpart, s.z, s.tickets + 1); break;
-    case 4: k_stream_downproj<4><<<grid, 256, 0, st>>>(h, A, M, d, r, slab, s.zpart, s.z, s.tickets + 1); break;
-    default: k_stream_downproj<8><<<grid, 256, 0, st>>>(h, A, M, d, r, slab, s.zpart, s.z, s.tickets + 1); break;
+    case 1: k_stream_downproj<1, 1024, 8><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z); break;
+    case 2: k_stream_downproj<2, 1024, 4><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z); break;
+    case 4: k_stream_downproj<4, 512, 8><<<grid, 512, 0, st>>>(h, A, M, d, r, s.z); break;
+    default: k_stream_downproj<8, 256, 8><<<grid, 256, 0, st>>>(h, A, M, d, r, s.z); break;
     }
     return cudaGetLastError();
 }
@@ -578,16 +634,16 @@ cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaS
     return cudaGetLastError();
 }
 
-template <int MT, int KG>
-static cudaError_t launch_head(const HeadParams& hp, size_t smem, bool pdl, cudaStream_t st)
+template <int MT, int U>
+static cudaError_t launch_head(const HeadParams& hp, const Geometry& g, bool pdl, cudaStream_t st)
 {
-    auto kern = k_stream_head<MT, KG>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto kern = k_stream_head<MT, U>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(hp.ncta);
-    cfg.blockDim = dim3(32 + 128 * KG + 32 * kEpiWarps);
-    cfg.dynamicSmemBytes = smem;
+    cfg.blockDim = dim3(g.threads);
+    cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -607,15 +663,15 @@ cudaError_t stream_head(const float* zT, const bf16* B, int M, int mt, int K, in
     HeadParams hp;
     hp.zT = zT; hp.B = B; hp.M = M; hp.K = K; hp.V = V; hp.k = k; hp.mode = mode;
     hp.ncta = g.ncta; hp.units_base = g.units_base; hp.units_rem = g.units_rem; hp.pass_units = g.pass_units;
-    hp.nstages = g.nstages; hp.pitch = g.pitch;
+    hp.ct = g.ct; hp.rg = g.rg; hp.kc = g.kc; hp.rec_words = g.rec_words; hp.merge_rows = g.merge_rows;
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     hp.wait_prev = after_producer_kernel ? 1 : 0;
     switch (mt) {
-    case 1: return launch_head<1, 4>(hp, g.smem, after_producer_kernel, st);
-    case 2: return launch_head<2, 4>(hp, g.smem, after_producer_kernel, st);
-    case 4: return launch_head<4, 4>(hp, g.smem, after_producer_kernel, st);
-    default: return launch_head<8, 2>(hp, g.smem, after_producer_kernel, st);
+    case 1: return launch_head<1, 16>(hp, g, after_producer_kernel, st);
+    case 2: return launch_head<2, 16>(hp, g, after_producer_kernel, st);
+    case 4: return launch_head<4, 8>(hp, g, after_producer_kernel, st);
+    default: return launch_head<8, 16>(hp, g, after_producer_kernel, st);
     }
 }
 
