@@ -44,58 +44,60 @@ struct HeadParams {
 // ends up with the j-th best.
 
 // One round: does this lane's head win?  The winner has the largest key, and among equal keys
-// the lowest id.  *any is false once no candidate is left.
-__device__ __forceinline__ bool round_winner(uint32_t hk, int hi, bool* any)
+// the lowest id (the second reduction runs only when keys tie).  With no candidate left the
+// "winner" is an empty entry (key 0, id kNoId).
+__device__ __forceinline__ bool round_winner(uint32_t hk, int hi)
 {
     const uint32_t wk = warp_max_u32(hk);
-    *any = wk != 0u;
-    const unsigned tied = __ballot_sync(0xffffffffu, hk == wk);
-    if (__popc(tied) == 1) return hk == wk;
-    const int wi = (int)warp_min_u32(hk == wk ? (uint32_t)hi : 0xffffffffu);
-    return hk == wk && hi == wi;
+    bool win = hk == wk;
+    const unsigned tied = __ballot_sync(0xffffffffu, win);
+    if (tied & (tied - 1)) {
+        const uint32_t wi = warp_min_u32(win ? (uint32_t)hi : 0xffffffffu);
+        win = win && (uint32_t)hi == wi;
+    }
+    return win;
 }
 
 // The winner of round j drops its head into out_k[j], out_i[j] (shared memory, one pair of
-// 32-entry arrays per warp); nothing but the pop of the winner's list sits between two rounds.
-// Entries j >= (number of candidates) are left as they were: callers clear the arrays first.
+// 32-entry arrays per warp), so nothing but the pop of the winner's list sits between two
+// rounds, and that pop is a select, not a branch.
 
 // Lists held in registers, NL entries per lane (unused entries: key 0, id kNoId).
 template <int NL>
 __device__ __forceinline__ void warp_topk_regs(uint32_t (&ck)[NL], int (&ci)[NL], int k, uint32_t* out_k, int* out_i)
 {
     for (int j = 0; j < k; ++j) {
-        bool any;
-        const bool win = round_winner(ck[0], ci[0], &any);
-        if (!any) break;
-        if (win) {
-            out_k[j] = ck[0];
-            out_i[j] = ci[0];
+        const bool win = round_winner(ck[0], ci[0]);
+        if (win) { out_k[j] = ck[0]; out_i[j] = ci[0]; }
 #pragma unroll
-            for (int s = 0; s + 1 < NL; ++s) { ck[s] = ck[s + 1]; ci[s] = ci[s + 1]; }
-            ck[NL - 1] = 0u;
-            ci[NL - 1] = kNoId;
-        }
+        for (int s = 0; s + 1 < NL; ++s) { ck[s] = win ? ck[s + 1] : ck[s]; ci[s] = win ? ci[s + 1] : ci[s]; }
+        ck[NL - 1] = win ? 0u : ck[NL - 1];
+        ci[NL - 1] = win ? kNoId : ci[NL - 1];
     }
 }
 
-// Lists held in shared memory: this lane's list is keys[0..len), ids[0..len).
+// Lists held in shared memory: this lane's list is keys[0..len), ids[0..len).  The entry after
+// the head is fetched ahead, so a pop never waits for shared memory.
 __device__ __forceinline__ void warp_topk_smem(const uint32_t* keys, const int* ids, int len, int k, uint32_t* out_k,
                                                int* out_i)
 {
     int pos = 0;
     uint32_t hk = len > 0 ? keys[0] : 0u;
     int hi = len > 0 ? ids[0] : kNoId;
+    uint32_t nk = len > 1 ? keys[1] : 0u;
+    int ni = len > 1 ? ids[1] : kNoId;
     for (int j = 0; j < k; ++j) {
-        bool any;
-        const bool win = round_winner(hk, hi, &any);
-        if (!any) break;
-        if (win) {
-            out_k[j] = hk;
-            out_i[j] = hi;
-            ++pos;
-            hk = pos < len ? keys[pos] : 0u;
-            hi = pos < len ? ids[pos] : kNoId;
-        }
+        const bool win = round_winner(hk, hi);
+        if (win) { out_k[j] = hk; out_i[j] = hi; }
+        pos += win ? 1 : 0;
+        hk = win ? nk : hk;
+        hi = win ? ni : hi;
+        const bool more = pos + 1 < len;
+        const int nx = more ? pos + 1 : 0;
+        const uint32_t tk = keys[len > 0 ? nx : 0];
+        const int ti = ids[len > 0 ? nx : 0];
+        nk = more ? tk : 0u;
+        ni = more ? ti : kNoId;
     }
 }
 
