@@ -45,6 +45,7 @@ extern "C" {
 #define SLIMSPEC_ERR_CUDA (-4)      /* a CUDA runtime call or a launch failed                  */
 #define SLIMSPEC_ERR_TIMEOUT (-5)   /* a bounded device-side wait ran out (see last_error)     */
 #define SLIMSPEC_ERR_NOMEM (-6)     /* device memory for scratch could not be allocated        */
+#define SLIMSPEC_ERR_STATIC_LIMIT (-7) /* beyond the fixed scratch of slimspec_head_topk_static */
 
 /* execution paths (slimspec_force_path) */
 #define SLIMSPEC_PATH_AUTO 0        /* chosen per (M, shapes) from measured timings            */
@@ -132,6 +133,39 @@ int slimspec_kernel_timing(slimspec_ctx* ctx, int enable);
  * milliseconds and their number (both host pointers, both required).
  */
 int slimspec_kernel_timing_read(slimspec_ctx* ctx, double* total_ms, long long* launches);
+
+/*
+ * The low-rank head with fused log-softmax / top-k for callers that cannot allocate device
+ * memory.  (The paper has no counterpart: this entry point exists for deployment only; it
+ * computes exactly what slimspec_head_topk computes on its streaming path.)
+ *
+ * Who needs it: code that runs where cudaMalloc / cudaFree are off limits -- inside a serving
+ * loop whose memory pool already owns the whole device, in a plugin whose host runtime forbids
+ * driver allocations on its worker threads, or in a latency-critical section that cannot take
+ * the device-wide synchronisation an allocation implies.  This call needs no context and calls
+ * no allocating routine: its scratch (the fp32 code z, the per-slab records, a ticket and an
+ * error word, about 0.8 MB) is a fixed device array inside the library image, held by every
+ * GPU that loads the library until the process exits.
+ *
+ * Limits, because that array has a fixed size: M <= SLIMSPEC_STATIC_MAX_M,
+ * r <= SLIMSPEC_STATIC_MAX_R, k <= SLIMSPEC_STATIC_MAX_K; larger values return
+ * SLIMSPEC_ERR_STATIC_LIMIT and launch nothing.  Shapes the streaming kernels do not take
+ * (V not a multiple of 8, r not a multiple of 16, pointers not 16-byte aligned) return
+ * SLIMSPEC_ERR_ALIGN.  h, A, B, out_ids, out_logprobs are device pointers with the layouts of
+ * slimspec_head_topk; the work is enqueued on `stream` without synchronising.
+ *
+ * The first call on a device looks up the device address of the array (once per device, with
+ * that device current); make that first call before any stream capture begins.
+ * All calls on a device share the one array, and it keeps the previous call's contents (the
+ * call clears the words that must start at zero).  Two calls whose kernels overlap on the GPU
+ * -- different streams, or several host threads -- race on it: serialise them.
+ */
+#define SLIMSPEC_STATIC_MAX_M 8
+#define SLIMSPEC_STATIC_MAX_R 8192
+#define SLIMSPEC_STATIC_MAX_K 32
+int slimspec_head_topk_static(const void* h, const void* A, const void* B,
+                              int M, int d, int r, int V, int k,
+                              int32_t* out_ids, float* out_logprobs, void* stream);
 
 /* Static description of a status code. */
 const char* slimspec_strerror(int status);

@@ -14,6 +14,8 @@ from . import build as _build
 
 OK = 0
 ERR_NULL, ERR_DIM, ERR_ALIGN, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = -1, -2, -3, -4, -5, -6
+ERR_STATIC_LIMIT = -7
+STATIC_MAX_M, STATIC_MAX_R, STATIC_MAX_K = 8, 8192, 32
 PATH_AUTO, PATH_GENERIC, PATH_STREAM, PATH_TENSOR = 0, 1, 2, 3
 MAX_K = 64
 
@@ -21,7 +23,7 @@ EXPORTS = [
     "slimspec_create", "slimspec_destroy", "slimspec_force_path", "slimspec_last_path",
     "slimspec_head_topk", "slimspec_head_topk_host", "slimspec_head_logits", "fullhead_topk",
     "slimspec_last_error", "slimspec_launch_count", "slimspec_strerror",
-    "slimspec_kernel_timing", "slimspec_kernel_timing_read",
+    "slimspec_kernel_timing", "slimspec_kernel_timing_read", "slimspec_head_topk_static",
 ]
 
 _lib = None
@@ -72,6 +74,8 @@ def load():
     lib.slimspec_kernel_timing_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double),
                                                 ctypes.POINTER(ctypes.c_longlong)]
     lib.slimspec_kernel_timing_read.restype = ci
+    lib.slimspec_head_topk_static.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, vp, vp, vp]
+    lib.slimspec_head_topk_static.restype = ci
     lib.slimspec_strerror.argtypes = [ci]
     lib.slimspec_strerror.restype = ctypes.c_char_p
     _lib = lib
@@ -209,3 +213,23 @@ class Context:
         if rc != OK:
             raise SlimSpecError(rc, "fullhead_topk")
         return out_ids, out_logprobs
+
+
+def slimspec_head_topk_static(h, A, B, k, out_ids, out_logprobs, stream=None):
+    """slimspec_head_topk_static of the C ABI: no context, no allocation (here neither: the
+    caller passes the output tensors).  For callers that must not allocate device memory --
+    a serving loop whose pool owns the device, a plugin under a runtime that forbids driver
+    allocations.  M <= 8, r <= 8192, k <= 32; calls that overlap on the GPU race on the
+    library's one static scratch array."""
+    M, d = h.shape
+    r, V = B.shape
+    _check_dev(h, torch.bfloat16, (M, d), "h")
+    _check_dev(A, torch.bfloat16, (d, r), "A")
+    _check_dev(B, torch.bfloat16, (r, V), "B")
+    _check_dev(out_ids, torch.int32, (M, k), "out_ids")
+    _check_dev(out_logprobs, torch.float32, (M, k), "out_logprobs")
+    rc = load().slimspec_head_topk_static(_ptr(h), _ptr(A), _ptr(B), M, d, r, V, k,
+                                          _ptr(out_ids), _ptr(out_logprobs), _stream(stream))
+    if rc != OK:
+        raise SlimSpecError(rc, "slimspec_head_topk_static")
+    return out_ids, out_logprobs

@@ -43,6 +43,7 @@ extern "C" const char* slimspec_strerror(int status)
     case SLIMSPEC_ERR_CUDA: return "CUDA runtime or launch error";
     case SLIMSPEC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case SLIMSPEC_ERR_NOMEM: return "out of device memory for scratch";
+    case SLIMSPEC_ERR_STATIC_LIMIT: return "M, r or k beyond the fixed scratch of slimspec_head_topk_static (8 rows, r 8192, k 32)";
     default: return "unknown status";
     }
 }
