@@ -28,7 +28,8 @@ struct slimspec_ctx {
 };
 static const int kTimingEvents = 256;
 
-static const int kMaxParts = 1024;     // most V slabs any kernel writes per row
+static const int kMaxParts = 256;      // most V slabs any kernel writes per row
+static const int kStreamMaxRows = 8;   // largest M the streaming path is chosen for
 static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
@@ -66,10 +67,22 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     c->s.max_parts = kMaxParts;
     const size_t mpad = (size_t)round_up(max_M, kRowPad);
     const size_t z_elems = mpad * (size_t)max_d;
-    const size_t part_elems = mpad * (size_t)kMaxParts * (size_t)round_up(2 + 2 * max_k, 4);   // records padded to 16 bytes
+    // split-V records, padded to 16 bytes: the streaming path writes <= 8 rows x 256 slabs, the
+    // tensor path 128 * nrb rows x (SMs / nrb) slabs
+    const int rec_k = max_k < 32 ? max_k : 32;
+    const size_t mpad128 = (size_t)round_up(max_M, 128);
+    const size_t part_elems = ((size_t)kRowPad * 256 + (size_t)(c->sm_count + 8) * 128 + mpad128) *
+                              (size_t)round_up(2 + 2 * rec_k, 4);
+    // K-split partial tiles of the tensor-core down-projection: one 128 x 128 fp32 tile per SM, or one split
+    size_t zpart_elems = (size_t)(c->sm_count + 12) * 128 * 128;
+    if (zpart_elems < mpad128 * (size_t)max_d) zpart_elems = mpad128 * (size_t)max_d;
     bool ok = true;
     ok = ok && cudaMalloc(&c->s.z, z_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.zb, mpad128 * (size_t)max_d * sizeof(bf16)) == cudaSuccess;
+    c->s.part_elems = part_elems;
+    c->s.zpart_elems = zpart_elems;
     ok = ok && cudaMalloc(&c->s.tickets, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.err, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->h_stage, (size_t)max_M * max_d * sizeof(bf16)) == cudaSuccess;
@@ -92,7 +105,7 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
 {
     if (!c) return;
     cudaDeviceSynchronize();
-    cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.tickets); cudaFree(c->s.err);
+    cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.tickets); cudaFree(c->s.err);
     cudaFree(c->s.logits); cudaFree(c->h_stage); cudaFree(c->ids_stage); cudaFree(c->lp_stage);
     if (c->ev0) {
         for (int i = 0; i < kTimingEvents; ++i) { cudaEventDestroy(c->ev0[i]); cudaEventDestroy(c->ev1[i]); }
@@ -213,8 +226,13 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
                         (mode == 0 || aligned16(logits));
     StreamPlan sp = stream_plan(M, d, K, V, mode == 0 ? k : 1, c->sm_count);
     const bool stream_ok = sp.ok && ptr_ok && (!lowrank || r % 16 == 0);
-    if (path == SLIMSPEC_PATH_AUTO) path = stream_ok ? SLIMSPEC_PATH_STREAM : SLIMSPEC_PATH_GENERIC;
-    if (path == SLIMSPEC_PATH_TENSOR) return SLIMSPEC_ERR_ALIGN;   // tensor path not built yet
+    const bool tensor_fits = tensor_ok(M, K, V, k, mode) && ptr_ok && (!lowrank || (d % 64 == 0 && r >= 64));
+    if (path == SLIMSPEC_PATH_AUTO) {
+        // FP32 FMAs keep up with HBM only for a few rows; beyond that the tensor cores take over
+        if (M > kStreamMaxRows && tensor_fits) path = SLIMSPEC_PATH_TENSOR;
+        else path = stream_ok ? SLIMSPEC_PATH_STREAM : (tensor_fits ? SLIMSPEC_PATH_TENSOR : SLIMSPEC_PATH_GENERIC);
+    }
+    if (path == SLIMSPEC_PATH_TENSOR && !tensor_fits) return SLIMSPEC_ERR_ALIGN;
     if (path == SLIMSPEC_PATH_STREAM && !stream_ok) return SLIMSPEC_ERR_ALIGN;
     c->last_path = path;
 
@@ -230,6 +248,22 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         CK(generic_upproj(c->s.z, Bm, M, K, V, lg, st));
         c->launches += 2;
         if (mode == 0) { CK(generic_softmax_topk(lg, M, V, k, ids, logprobs, st)); c->launches += 1; }
+        return SLIMSPEC_OK;
+    }
+
+    if (path == SLIMSPEC_PATH_TENSOR) {
+        int n = 0;
+        const bf16* X = h;
+        if (lowrank) {
+            cudaError_t e0 = tensor_downproj(h, A, M, d, r, c->s, c->sm_count, &n, st);
+            c->launches += n;
+            n = 0;
+            if (e0 != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
+            X = c->s.zb;
+        }
+        cudaError_t e = tensor_head(X, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, &n, st);
+        c->launches += n;
+        if (e != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         return SLIMSPEC_OK;
     }
 

@@ -14,7 +14,11 @@ typedef __nv_bfloat16 bf16;
 // Layout in the context's scratch: float pm[P], ps[P], pv[P][k]; int pi[P][k] per row.
 struct Scratch {
     float* z;            // fp32 code (or widened h); generic path [M][K], streaming path transposed [K][mt]
+    bf16* zb;            // bf16 code [M][r] for the tensor-core path
+    float* zpart;        // K-split partial tiles of the tensor-core down-projection
+    size_t zpart_elems;
     float* part;         // split-V partial records
+    size_t part_elems;
     unsigned int* tickets;  // arrival counters (self-resetting)
     int* err;            // device error word
     float* logits;       // generic path only: M x V fp32, grown on demand
@@ -46,5 +50,15 @@ cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaS
 cudaError_t stream_head(const float* z, const bf16* B, int M, int mt, int K, int V, int k, int mode,
                         int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
                         bool after_producer_kernel, cudaStream_t st);
+
+// ---- tensor-core path (larger M) ------------------------------------------------------
+// Shapes the tcgen05 kernels take: K a multiple of 64, N a multiple of 8 and >= 64, k <= 32 in top-k mode.
+bool tensor_ok(int M, int K, int N, int k, int mode);
+// z (bf16 [M][r], in s.zb) = h A.
+cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, const Scratch& s, int sm_count,
+                            int* launches, cudaStream_t st);
+// X W with X bf16 [M][K], W bf16 [K][N]; mode 0: fused log-softmax / top-k, mode 1: raw fp32 logits.
+cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
+                        float* logprobs, float* logits, const Scratch& s, int sm_count, int* launches, cudaStream_t st);
 
 }  // namespace slimspec

@@ -1,0 +1,435 @@
+// Tensor-core path for larger M: out = X W with X[M][K] (rows on the MMA's M side, K-major) and
+// W[K][N] (N-major), bf16 inputs, fp32 accumulation in tensor memory (tcgen05).
+//   down-projection  z = h A      X = h, W = A, split over K, fp32 partial tiles -> k_tc_reduce_z
+//   up-projection    logits = z B X = z (bf16), W = B, fused online log-softmax / top-k epilogue
+//   full-rank head   logits = h W X = h, W = W, same epilogue
+// (Section 4.1; the softmax of Section 3.2 and the candidate selection.)
+//
+// One CTA per SM, six warps: warp 0 feeds a ring of shared-memory stages by TMA, one thread of
+// warp 1 issues the MMAs (128 rows x NV columns x 16 per instruction) into one of two
+// accumulator buffers in tensor memory, warps 2-5 read the finished buffer (a thread per row) and
+// keep that row's running max / sum-exp / top-k while the next tile's MMAs run.
+#include "kernels.h"
+#include "ptx.cuh"
+#include <cuda.h>
+#include <float.h>
+#include <string.h>
+
+namespace slimspec {
+
+static constexpr int kTcRows = 128;          // rows per tile = MMA M
+static constexpr int kTcKChunk = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
+static constexpr int kTcThreads = 192;
+static constexpr int kTcMaxK = 32;           // top-k entries a row keeps
+static constexpr int kTcNoId = 0x7fffffff;
+static constexpr float kLog2e = 1.4426950408889634f;
+
+struct alignas(64) TcParams {
+    CUtensorMap mapX;       // X[M][K]: box 64 (K) x 128 rows, 128-byte swizzle
+    CUtensorMap mapW;       // W[K][N]: box 64 (N) x 64 (K), 128-byte swizzle
+    int M, K, N;
+    int nrb, nct, nks;      // row blocks, column tiles, K splits
+    int chunks_per_split;   // K chunks of 64 per split
+    int gct;                // CTAs that share one (row block, split); column tiles go round-robin
+    int mode;               // 0: top-k records, 1: fp32 out[M][N], 2: fp32 partial out[nks][nrb*128][N]
+    int k;
+    int rec_words;
+    float* out;
+    float* part;            // records [M][gct][rec_words]
+    int* err;
+};
+
+// Insert (key, id) into a row's list of the k best (keys descending; of equal keys the earlier,
+// lower id stays in front).  thr is the key of the k-th entry once the list is full, else 0.
+__device__ __noinline__ void topk_insert(uint32_t* lk, int* li, int& cnt, uint32_t& thr, int k, uint32_t key, int id)
+{
+    int pos = cnt < k ? cnt : k - 1;
+    while (pos > 0 && lk[pos - 1] < key) {
+        lk[pos] = lk[pos - 1];
+        li[pos] = li[pos - 1];
+        --pos;
+    }
+    lk[pos] = key;
+    li[pos] = id;
+    cnt = cnt < k ? cnt + 1 : k;
+    thr = cnt == k ? lk[k - 1] : 0u;
+}
+
+// ------------------------------------------------------------------------------------------
+template <int NV>
+__global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant__ TcParams p)
+{
+    constexpr int NS = (NV == 256) ? 4 : 6;                 // ring stages
+    constexpr int X_BYTES = kTcRows * kTcKChunk * 2;        // 16 KB
+    constexpr int WBOX_BYTES = kTcKChunk * 64 * 2;          // 8 KB: 64 k x 64 columns
+    constexpr int W_BYTES = WBOX_BYTES * (NV / 64);
+    constexpr int STAGE = X_BYTES + W_BYTES;
+    // instruction descriptor: D fp32, A and B bf16, A K-major, B MN-major, N = NV, M = 128
+    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                               ((uint32_t)(NV >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
+
+    extern __shared__ unsigned char smem_raw[];
+    __shared__ uint64_t full[NS], empty[NS], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    unsigned char* stages = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    volatile int* abort_flag = &abort_s;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x;
+    const int rb = cta % p.nrb;
+    const int rest = cta / p.nrb;
+    const int ks = rest % p.nks;
+    const int cg = rest / p.nks;                 // position among the CTAs of this (row block, split)
+    const int cps = p.chunks_per_split;
+    const int ntiles = cg < p.nct ? (p.nct - cg + p.gct - 1) / p.gct : 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+        abort_s = 0;
+        mbar_fence_init();
+        prefetch_tensor_map(&p.mapX);
+        prefetch_tensor_map(&p.mapW);
+    }
+    if (warp == 1) tmem_alloc(&tmem_base_s, 2 * NV);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (warp == 0) {
+        // ================= producer: one thread issues the TMA loads =================
+        if (lane == 0) {
+            int it = 0;
+            bool alive = true;
+            for (int t = 0; t < ntiles && alive; ++t) {
+                const int ct = cg + t * p.gct;
+                for (int c = 0; c < cps; ++c, ++it) {
+                    const int s = it % NS, use = it / NS;
+                    if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, p.err, ERR_WAIT_EMPTY)) { alive = false; break; }
+                    unsigned char* st = stages + (size_t)s * STAGE;
+                    mbar_arrive_expect_tx(&full[s], STAGE);
+                    const int kx = (ks * cps + c) * kTcKChunk;
+                    tma_load_2d(st, &p.mapX, kx, rb * kTcRows, &full[s]);
+#pragma unroll
+                    for (int i = 0; i < NV / 64; ++i)
+                        tma_load_2d(st + X_BYTES + i * WBOX_BYTES, &p.mapW, ct * NV + i * 64, kx, &full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            int it = 0;
+            bool alive = true;
+            for (int t = 0; t < ntiles && alive; ++t) {
+                const int buf = t & 1;
+                if (t >= 2 && !mbar_wait(&acc_empty[buf], ((t >> 1) - 1) & 1, abort_flag, p.err, ERR_WAIT_FREE)) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NV);
+                for (int c = 0; c < cps; ++c, ++it) {
+                    const int s = it % NS, use = it / NS;
+                    if (!mbar_wait(&full[s], use & 1, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t xa = smem_u32(stages + (size_t)s * STAGE);
+                    const uint64_t a_desc = tc_smem_desc_sw128(xa, 16, 1024);
+                    const uint64_t b_desc = tc_smem_desc_sw128(xa + X_BYTES, WBOX_BYTES, 1024);
+#pragma unroll
+                    for (int j = 0; j < kTcKChunk / 16; ++j) {
+                        // 16 of K per instruction: 32 bytes along a K-major row, two 8-row groups of the N-major tile
+                        tc_mma_bf16(d_tmem, a_desc + (uint64_t)(j * 2), b_desc + (uint64_t)(j * 128), IDESC,
+                                    (c > 0 || j > 0) ? 1u : 0u);
+                    }
+                    tc_commit(&empty[s]);
+                }
+                if (alive) tc_commit(&acc_full[buf]);
+            }
+        }
+    } else {
+        // ================= epilogue: thread = row =================
+        const int quarter = warp & 3;                        // the lane quarter this warp may read
+        const int row = quarter * 32 + lane;
+        const int m = rb * kTcRows + row;
+        const bool live = m < p.M;
+        const int k = p.k;
+        float run_max = -FLT_MAX, run_sum = 0.f;
+        uint32_t lk[kTcMaxK];
+        int li[kTcMaxK];
+        int cnt = 0;
+        uint32_t thr = 0u;                                   // key of the k-th best once the list is full
+        bool alive = true;
+        for (int t = 0; t < ntiles && alive; ++t) {
+            const int buf = t & 1;
+            const int ct = cg + t * p.gct;
+            if (!mbar_wait(&acc_full[buf], (t >> 1) & 1, abort_flag, p.err, ERR_WAIT_ACC)) { alive = false; break; }
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NV);
+#pragma unroll 1
+            for (int c0 = 0; c0 < NV; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32x32(taddr + (uint32_t)c0, v);
+                tmem_ld_wait();
+                const int col0 = ct * NV + c0;
+                const int nvalid = min(32, p.N - col0);      // same for every thread
+                if (nvalid <= 0 || !live) continue;
+                if (p.mode != 0) {
+                    const size_t orow = (p.mode == 2) ? ((size_t)ks * p.nrb * kTcRows + m) : (size_t)m;
+                    float* dst = p.out + orow * p.N + col0;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        if (e < nvalid)      // N is a multiple of 8, so a group of four is all in or all out
+                            *reinterpret_cast<float4*>(dst + e) =
+                                make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
+                                            __uint_as_float(v[e + 3]));
+                    }
+                    continue;
+                }
+                // online softmax
+                float cmax = -FLT_MAX;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) cmax = fmaxf(cmax, e < nvalid ? __uint_as_float(v[e]) : -FLT_MAX);
+                if (cmax > run_max) {
+                    run_sum *= exp2f((run_max - cmax) * kLog2e);
+                    run_max = cmax;
+                }
+                const float mb = run_max * kLog2e;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    s0 += e < nvalid ? exp2f(fmaf(__uint_as_float(v[e]), kLog2e, -mb)) : 0.f;
+                    s1 += e + 1 < nvalid ? exp2f(fmaf(__uint_as_float(v[e + 1]), kLog2e, -mb)) : 0.f;
+                }
+                run_sum += s0 + s1;
+                // top-k: ids arrive in ascending order, so a candidate must beat the k-th key strictly
+                if (f2key(cmax) > thr) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const uint32_t key = f2key(__uint_as_float(v[e]));
+                        if (e < nvalid && key > thr) topk_insert(lk, li, cnt, thr, k, key, col0 + e);
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&acc_empty[buf]);
+        }
+        if (alive && live && p.mode == 0) {
+            float* rec = p.part + ((size_t)m * p.gct + cg) * p.rec_words;
+            rec[0] = run_max;
+            rec[1] = run_sum;
+            for (int j = 0; j < k; ++j) {
+                rec[2 + j] = __uint_as_float(j < cnt ? lk[j] : 0u);
+                rec[2 + k + j] = __int_as_float(j < cnt ? li[j] : kTcNoId);
+            }
+        }
+    }
+    // ---- teardown: every role is past its last use of tensor memory
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 1) tmem_dealloc(tmem_base, 2 * NV);
+}
+
+// ------------------------------------------------------------------------------------------
+// z = sum of the K-split partial tiles, rounded once to bf16.
+__global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad, int M, int r, bf16* __restrict__ z)
+{
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= M * r) return;
+    const int m = e / r, j = e - m * r;
+    float acc = 0.f;
+    for (int s0 = 0; s0 < nks; s0 += 8) {
+        float t[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) t[q] = (s0 + q < nks) ? __ldcg(part + ((size_t)(s0 + q) * mpad + m) * r + j) : 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc += t[q];
+    }
+    z[e] = __float2bfloat16_rn(acc);
+}
+
+// ------------------------------------------------------------------------------------------
+// Merge the P per-slab records of each row: one warp per row, a lane owns up to 8 slab lists.
+__global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part, int M, int P, int RW, int k,
+                                                  int32_t* __restrict__ ids, float* __restrict__ logprobs)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (m >= M) return;
+    const float* rows = part + (size_t)m * P * RW;
+    float gm = -FLT_MAX;
+    for (int s = lane; s < P; s += 32) gm = fmaxf(gm, __ldcg(rows + (size_t)s * RW));
+    gm = warp_max(gm);
+    float gs = 0.f;
+    for (int s = lane; s < P; s += 32)
+        gs += __ldcg(rows + (size_t)s * RW + 1) * __expf(__ldcg(rows + (size_t)s * RW) - gm);
+    gs = warp_sum(gs);
+    const float lse = gm + __logf(gs);
+    uint32_t hk[8];
+    int hi[8], hp[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int s = lane + 32 * q;
+        hp[q] = 0;
+        hk[q] = (s < P) ? __float_as_uint(__ldcg(rows + (size_t)s * RW + 2)) : 0u;
+        hi[q] = (s < P) ? __float_as_int(__ldcg(rows + (size_t)s * RW + 2 + k)) : kTcNoId;
+    }
+    uint32_t ok = 0;
+    int oi = kTcNoId;
+    for (int j = 0; j < k; ++j) {
+        uint32_t bk = hk[0];
+        int bi = hi[0], bs = 0;
+#pragma unroll
+        for (int q = 1; q < 8; ++q) {
+            const bool better = hk[q] > bk || (hk[q] == bk && hi[q] < bi);
+            bk = better ? hk[q] : bk;
+            bi = better ? hi[q] : bi;
+            bs = better ? q : bs;
+        }
+        const uint32_t wk = warp_max_u32(bk);
+        const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
+        const bool win = (bk == wk) && ((uint32_t)bi == wi);
+        if (win && wk != 0u) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (q == bs) {
+                    const int s = lane + 32 * q;
+                    const int np = hp[q] + 1;
+                    hp[q] = np;
+                    hk[q] = (np < k) ? __float_as_uint(__ldcg(rows + (size_t)s * RW + 2 + np)) : 0u;
+                    hi[q] = (np < k) ? __float_as_int(__ldcg(rows + (size_t)s * RW + 2 + k + np)) : kTcNoId;
+                }
+            }
+        }
+        if (lane == j) { ok = wk; oi = (int)wi; }
+    }
+    if (lane < k) {
+        ids[(size_t)m * k + lane] = oi;
+        logprobs[(size_t)m * k + lane] = key2f(ok) - lse;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)ptr;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] (cols contiguous), box = box_cols x box_rows, 128-byte swizzle, zero fill
+static bool make_map(CUtensorMap* map, const void* base, int rows, int cols, int box_cols, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t es[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tensor_ok(int M, int K, int N, int k, int mode)
+{
+    if (M < 1 || K < kTcKChunk || K % kTcKChunk != 0 || N % 8 != 0 || N < 64) return false;
+    if (mode == 0 && (k < 1 || k > kTcMaxK)) return false;
+    return true;
+}
+
+template <int NV>
+static cudaError_t launch_gemm(const TcParams& p, int grid, cudaStream_t st)
+{
+    constexpr int NS = (NV == 256) ? 4 : 6;
+    constexpr int STAGE = kTcRows * kTcKChunk * 2 + kTcKChunk * NV * 2;
+    const size_t smem = (size_t)NS * STAGE + 1024;
+    auto kern = k_tc_gemm<NV>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kTcThreads, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+// out = X W through the tensor cores.  mode 0: top-k records then merge into ids / logprobs;
+// mode 1: fp32 logits.  X is bf16 [M][K], W bf16 [K][N].
+cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
+                        float* logprobs, float* logits, const Scratch& s, int sm_count, int* launches, cudaStream_t st)
+{
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    if (!make_map(&p.mapX, X, M, K, kTcKChunk, kTcRows) || !make_map(&p.mapW, W, K, N, 64, kTcKChunk))
+        return cudaErrorInvalidValue;
+    p.M = M; p.K = K; p.N = N;
+    p.nrb = (M + kTcRows - 1) / kTcRows;
+    const int nv = (p.nrb == 1) ? 128 : 256;
+    p.nct = (N + nv - 1) / nv;
+    p.nks = 1;
+    p.chunks_per_split = K / kTcKChunk;
+    p.gct = sm_count / p.nrb;
+    if (p.gct < 1) p.gct = 1;
+    if (p.gct > p.nct) p.gct = p.nct;
+    if (p.gct > 256) p.gct = 256;
+    p.mode = mode;
+    p.k = k;
+    p.rec_words = (2 + 2 * k + 3) / 4 * 4;
+    p.out = logits;
+    p.part = s.part;
+    p.err = s.err;
+    if (mode == 0 && (size_t)M * p.gct * p.rec_words > s.part_elems) return cudaErrorInvalidValue;
+    const int grid = p.gct * p.nrb;
+    cudaError_t e = (nv == 128) ? launch_gemm<128>(p, grid, st) : launch_gemm<256>(p, grid, st);
+    if (e != cudaSuccess) return e;
+    *launches += 1;
+    if (mode == 0) {
+        k_tc_merge<<<(M + 7) / 8, 256, 0, st>>>(s.part, M, p.gct, p.rec_words, k, ids, logprobs);
+        *launches += 1;
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+// z (bf16, [M][r]) = h A through the tensor cores: K-split partial tiles, then one reduction.
+cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, const Scratch& s, int sm_count,
+                            int* launches, cudaStream_t st)
+{
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    if (!make_map(&p.mapX, h, M, d, kTcKChunk, kTcRows) || !make_map(&p.mapW, A, d, r, 64, kTcKChunk))
+        return cudaErrorInvalidValue;
+    p.M = M; p.K = d; p.N = r;
+    p.nrb = (M + kTcRows - 1) / kTcRows;
+    p.nct = (r + 127) / 128;
+    const int chunks = d / kTcKChunk;
+    // as many K splits as fill the SMs once, each a whole number of chunks
+    int nks = sm_count / (p.nrb * p.nct);
+    if (nks < 1) nks = 1;
+    if (nks > chunks) nks = chunks;
+    while (chunks % nks != 0) --nks;
+    p.nks = nks;
+    p.chunks_per_split = chunks / nks;
+    p.gct = p.nct;
+    p.mode = 2;
+    p.out = s.zpart;
+    p.err = s.err;
+    const size_t need = (size_t)nks * p.nrb * kTcRows * r;
+    if (need > s.zpart_elems) return cudaErrorInvalidValue;
+    cudaError_t e = launch_gemm<128>(p, p.nrb * p.nct * nks, st);
+    if (e != cudaSuccess) return e;
+    const int n = M * r;
+    k_tc_reduce_z<<<(n + 255) / 256, 256, 0, st>>>(s.zpart, nks, p.nrb * kTcRows, M, r, s.zb);
+    *launches += 2;
+    return cudaGetLastError();
+}
+
+}  // namespace slimspec
