@@ -81,6 +81,9 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zb, mpad128 * (size_t)max_d * sizeof(bf16)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.smax, 64 * mpad128 * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.thr0, mpad128 * sizeof(uint32_t)) == cudaSuccess;
+    c->s.smax_elems = 64 * mpad128;
     c->s.part_elems = part_elems;
     c->s.zpart_elems = zpart_elems;
     ok = ok && cudaMalloc(&c->s.tickets, 4096 * sizeof(unsigned int)) == cudaSuccess;
@@ -105,7 +108,7 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
 {
     if (!c) return;
     cudaDeviceSynchronize();
-    cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.tickets); cudaFree(c->s.err);
+    cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.smax); cudaFree(c->s.thr0); cudaFree(c->s.tickets); cudaFree(c->s.err);
     cudaFree(c->s.logits); cudaFree(c->h_stage); cudaFree(c->ids_stage); cudaFree(c->lp_stage);
     if (c->ev0) {
         for (int i = 0; i < kTimingEvents; ++i) { cudaEventDestroy(c->ev0[i]); cudaEventDestroy(c->ev1[i]); }

@@ -17,6 +17,9 @@ struct Scratch {
     bf16* zb;            // bf16 code [M][r] for the tensor-core path
     float* zpart;        // K-split partial tiles of the tensor-core down-projection
     size_t zpart_elems;
+    uint32_t* smax;      // tensor path: per-row maxima of the sample tiles [64][M padded to 128]
+    size_t smax_elems;
+    uint32_t* thr0;      // tensor path: per-row starting bound of the top-k lists
     float* part;         // split-V partial records
     size_t part_elems;
     unsigned int* tickets;  // arrival counters (self-resetting)

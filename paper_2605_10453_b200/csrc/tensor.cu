@@ -31,7 +31,10 @@ struct alignas(64) TcParams {
     int nrb, nct, nks;      // row blocks, column tiles, K splits
     int chunks_per_split;   // K chunks of 64 per split
     int gct;                // CTAs that share one (row block, split); column tiles go round-robin
-    int mode;               // 0: top-k records, 1: fp32 out[M][N], 2: fp32 partial out[nks][nrb*128][N]
+    int mode;               // 0: top-k records, 1: fp32 out[M][N], 2: fp32 partial out[nks][nrb*128][N],
+                            // 3: per-row maximum of each tile, as a key, to smax[tile][nrb*128]
+    uint32_t* smax;         // mode 3 output
+    const uint32_t* thr0;   // mode 0: per-row lower bound (key - 1) of the k-th largest logit, or null
     int k;
     int rec_words;
     float* out;
@@ -40,8 +43,10 @@ struct alignas(64) TcParams {
 };
 
 // Insert (key, id) into a row's list of the k best (keys descending; of equal keys the earlier,
-// lower id stays in front).  thr is the key of the k-th entry once the list is full, else 0.
-__device__ __noinline__ void topk_insert(uint32_t* lk, int* li, int& cnt, uint32_t& thr, int k, uint32_t key, int id)
+// lower id stays in front).  thr is the key of the k-th entry once the list is full, else the
+// row's starting bound thr0: only keys above thr are ever offered.
+__device__ __noinline__ void topk_insert(uint32_t* lk, int* li, int& cnt, uint32_t& thr, int k, uint32_t key, int id,
+                                         uint32_t thr0)
 {
     int pos = cnt < k ? cnt : k - 1;
     while (pos > 0 && lk[pos - 1] < key) {
@@ -52,7 +57,7 @@ __device__ __noinline__ void topk_insert(uint32_t* lk, int* li, int& cnt, uint32
     lk[pos] = key;
     li[pos] = id;
     cnt = cnt < k ? cnt + 1 : k;
-    thr = cnt == k ? lk[k - 1] : 0u;
+    thr = cnt == k ? lk[k - 1] : thr0;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -157,7 +162,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         uint32_t lk[kTcMaxK];
         int li[kTcMaxK];
         int cnt = 0;
-        uint32_t thr = 0u;                                   // key of the k-th best once the list is full
+        // Candidates must beat thr: the key of the k-th best once the list is full, before that a
+        // bound known to lie below the row's k-th largest logit (from a sample of the vocabulary).
+        const uint32_t thr0 = (p.mode == 0 && p.thr0 != nullptr && live) ? __ldg(p.thr0 + m) : 0u;
+        uint32_t thr = thr0;
         bool alive = true;
         for (int t = 0; t < ntiles && alive; ++t) {
             const int buf = t & 1;
@@ -165,6 +173,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             if (!mbar_wait(&acc_full[buf], (t >> 1) & 1, abort_flag, p.err, ERR_WAIT_ACC)) { alive = false; break; }
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NV);
+            float tile_max = -FLT_MAX;
 #pragma unroll 1
             for (int c0 = 0; c0 < NV; c0 += 32) {
                 uint32_t v[32];
@@ -173,6 +182,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 const int col0 = ct * NV + c0;
                 const int nvalid = min(32, p.N - col0);      // same for every thread
                 if (nvalid <= 0 || !live) continue;
+                if (p.mode == 3) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) tile_max = fmaxf(tile_max, e < nvalid ? __uint_as_float(v[e]) : -FLT_MAX);
+                    continue;
+                }
                 if (p.mode != 0) {
                     const size_t orow = (p.mode == 2) ? ((size_t)ks * p.nrb * kTcRows + m) : (size_t)m;
                     float* dst = p.out + orow * p.N + col0;
@@ -206,10 +220,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 32; ++e) {
                         const uint32_t key = f2key(__uint_as_float(v[e]));
-                        if (e < nvalid && key > thr) topk_insert(lk, li, cnt, thr, k, key, col0 + e);
+                        if (e < nvalid && key > thr) topk_insert(lk, li, cnt, thr, k, key, col0 + e, thr0);
                     }
                 }
             }
+            if (p.mode == 3 && live) p.smax[(size_t)ct * p.nrb * kTcRows + m] = f2key(tile_max);
             tc_fence_before_sync();
             mbar_arrive(&acc_empty[buf]);
         }
@@ -246,6 +261,27 @@ __global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad,
         for (int q = 0; q < 8; ++q) acc += t[q];
     }
     z[e] = __float2bfloat16_rn(acc);
+}
+
+// ------------------------------------------------------------------------------------------
+// thr0[m] = (k-th largest of the row's nst sample-tile maxima) - 1, as a key: at least k logits
+// of the row are >= that maximum, so the row's k-th largest logit is too.  One warp per row,
+// nst <= 64.  Equal maxima are counted once, which only lowers the bound.  0 if nst < k.
+__global__ void __launch_bounds__(256) k_tc_thr0(const uint32_t* __restrict__ smax, int nst, int mpad, int M, int k,
+                                                 uint32_t* __restrict__ thr0)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m = blockIdx.x * (blockDim.x >> 5) + warp;
+    if (m >= M) return;
+    uint32_t a = lane < nst ? __ldcg(smax + (size_t)lane * mpad + m) : 0u;
+    uint32_t b = lane + 32 < nst ? __ldcg(smax + (size_t)(lane + 32) * mpad + m) : 0u;
+    if (b > a) { const uint32_t t = a; a = b; b = t; }
+    uint32_t kth = 0u;
+    for (int j = 0; j < k; ++j) {
+        kth = warp_max_u32(a);
+        if (a == kth) { a = b; b = 0u; }
+    }
+    if (lane == 0) thr0[m] = (nst >= k && kth > 0u) ? kth - 1u : 0u;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -387,8 +423,29 @@ cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k
     p.part = s.part;
     p.err = s.err;
     if (mode == 0 && (size_t)M * p.gct * p.rec_words > s.part_elems) return cudaErrorInvalidValue;
+    cudaError_t e;
+    if (mode == 0) {
+        // A bound below each row's k-th largest logit, from the first sample tiles of the vocabulary:
+        // it keeps the per-row candidate lists of the main pass almost idle.
+        int nst = 2 * k > 32 ? 2 * k : 32;
+        if (nst > p.nct) nst = p.nct;
+        if (nst >= k && (size_t)nst * p.nrb * kTcRows <= s.smax_elems) {
+            TcParams q = p;
+            q.mode = 3;
+            q.nct = nst;
+            q.gct = nst;
+            q.smax = s.smax;
+            e = (nv == 128) ? launch_gemm<128>(q, nst * p.nrb, st) : launch_gemm<256>(q, nst * p.nrb, st);
+            if (e != cudaSuccess) return e;
+            k_tc_thr0<<<(M + 7) / 8, 256, 0, st>>>(s.smax, nst, p.nrb * kTcRows, M, k, s.thr0);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+            *launches += 2;
+            p.thr0 = s.thr0;
+        }
+    }
     const int grid = p.gct * p.nrb;
-    cudaError_t e = (nv == 128) ? launch_gemm<128>(p, grid, st) : launch_gemm<256>(p, grid, st);
+    e = (nv == 128) ? launch_gemm<128>(p, grid, st) : launch_gemm<256>(p, grid, st);
     if (e != cudaSuccess) return e;
     *launches += 1;
     if (mode == 0) {
