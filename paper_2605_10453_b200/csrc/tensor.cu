@@ -42,22 +42,29 @@ struct alignas(64) TcParams {
     int* err;
 };
 
-// Insert (key, id) into a row's list of the k best (keys descending; of equal keys the earlier,
-// lower id stays in front).  thr is the key of the k-th entry once the list is full, else the
-// row's starting bound thr0: only keys above thr are ever offered.
-__device__ __noinline__ void topk_insert(uint32_t* lk, int* li, int& cnt, uint32_t& thr, int k, uint32_t key, int id,
-                                         uint32_t thr0)
+// Insert (value, id) into a row's list of the k best (values descending; of equal values the
+// earlier, lower id stays in front).  Returns the new threshold a candidate has to beat: the k-th
+// value once the list is full, else the row's starting bound thr0.
+__device__ __forceinline__ float topk_insert(float* lv, int* li, int& cnt, int k, float val, int id, float thr0)
 {
     int pos = cnt < k ? cnt : k - 1;
-    while (pos > 0 && lk[pos - 1] < key) {
-        lk[pos] = lk[pos - 1];
+    if (cnt == k && !(val > lv[k - 1])) return lv[k - 1];
+    while (pos > 0 && lv[pos - 1] < val) {
+        lv[pos] = lv[pos - 1];
         li[pos] = li[pos - 1];
         --pos;
     }
-    lk[pos] = key;
+    lv[pos] = val;
     li[pos] = id;
     cnt = cnt < k ? cnt + 1 : k;
-    thr = cnt == k ? lk[k - 1] : thr0;
+    return cnt == k ? lv[k - 1] : thr0;
+}
+
+__device__ __forceinline__ float ex2_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -159,13 +166,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         const bool live = m < p.M;
         const int k = p.k;
         float run_max = -FLT_MAX, run_sum = 0.f;
-        uint32_t lk[kTcMaxK];
+        float lv[kTcMaxK];
         int li[kTcMaxK];
         int cnt = 0;
-        // Candidates must beat thr: the key of the k-th best once the list is full, before that a
-        // bound known to lie below the row's k-th largest logit (from a sample of the vocabulary).
-        const uint32_t thr0 = (p.mode == 0 && p.thr0 != nullptr && live) ? __ldg(p.thr0 + m) : 0u;
-        uint32_t thr = thr0;
+        // Candidates must beat thr: the k-th best value once the list is full, before that a bound
+        // known to lie below the row's k-th largest logit (from a sample of the vocabulary).
+        const uint32_t thr0_key = (p.mode == 0 && p.thr0 != nullptr && live) ? __ldg(p.thr0 + m) : 0u;
+        const float thr0 = thr0_key != 0u ? key2f(thr0_key) : -FLT_MAX;      // key 0: no bound
+        float thr = thr0;
         bool alive = true;
         for (int t = 0; t < ntiles && alive; ++t) {
             const int buf = t & 1;
@@ -199,29 +207,57 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                     }
                     continue;
                 }
-                // online softmax
-                float cmax = -FLT_MAX;
+                // ---- online softmax and candidate filter; four independent chains keep the one
+                // warp of this scheduler busy.  Columns past N (last tile only) count as -FLT_MAX.
+                float x[32];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) cmax = fmaxf(cmax, e < nvalid ? __uint_as_float(v[e]) : -FLT_MAX);
+                for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]);
+                if (nvalid < 32) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x[e] = e < nvalid ? x[e] : -FLT_MAX;
+                }
+                float m8[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    m8[q] = x[q * 8];
+#pragma unroll
+                    for (int e = 1; e < 8; ++e) m8[q] = fmaxf(m8[q], x[q * 8 + e]);
+                }
+                const float cmax = fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3]));
                 if (cmax > run_max) {
-                    run_sum *= exp2f((run_max - cmax) * kLog2e);
+                    run_sum *= ex2_fast((run_max - cmax) * kLog2e);
                     run_max = cmax;
                 }
                 const float mb = run_max * kLog2e;
-                float s0 = 0.f, s1 = 0.f;
+                float sacc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    s0 += e < nvalid ? exp2f(fmaf(__uint_as_float(v[e]), kLog2e, -mb)) : 0.f;
-                    s1 += e + 1 < nvalid ? exp2f(fmaf(__uint_as_float(v[e + 1]), kLog2e, -mb)) : 0.f;
-                }
-                run_sum += s0 + s1;
-                // top-k: ids arrive in ascending order, so a candidate must beat the k-th key strictly
-                if (f2key(cmax) > thr) {
+                for (int e = 0; e < 32; ++e) sacc[e & 3] += ex2_fast(fmaf(x[e], kLog2e, -mb));
+                run_sum += (sacc[0] + sacc[1]) + (sacc[2] + sacc[3]);
+                // top-k: ids arrive in ascending order, so a candidate must beat the threshold strictly.
+                // Only groups of eight whose maximum passes are looked at; what passes is parked and
+                // inserted after the scan, so the scan itself is compare-and-branch only.
+                if (cmax > thr) {
+                    float pend_v[8];
+                    int pend_i[8];
+                    int np = 0;
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const uint32_t key = f2key(__uint_as_float(v[e]));
-                        if (e < nvalid && key > thr) topk_insert(lk, li, cnt, thr, k, key, col0 + e, thr0);
+                    for (int q = 0; q < 4; ++q) {
+                        if (m8[q] > thr) {
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                if (x[q * 8 + e] > thr) {
+                                    if (np == 8) {       // rare: flush the parked candidates
+                                        for (int j = 0; j < 8; ++j) thr = topk_insert(lv, li, cnt, k, pend_v[j], pend_i[j], thr0);
+                                        np = 0;
+                                    }
+                                    pend_v[np] = x[q * 8 + e];
+                                    pend_i[np] = col0 + q * 8 + e;
+                                    ++np;
+                                }
+                            }
+                        }
                     }
+                    for (int j = 0; j < np; ++j) thr = topk_insert(lv, li, cnt, k, pend_v[j], pend_i[j], thr0);
                 }
             }
             if (p.mode == 3 && live) p.smax[(size_t)ct * p.nrb * kTcRows + m] = f2key(tile_max);
@@ -233,7 +269,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             rec[0] = run_max;
             rec[1] = run_sum;
             for (int j = 0; j < k; ++j) {
-                rec[2 + j] = __uint_as_float(j < cnt ? lk[j] : 0u);
+                rec[2 + j] = __uint_as_float(j < cnt ? f2key(lv[j] + 0.f) : 0u);      // -0 and +0 rank alike
                 rec[2 + k + j] = __int_as_float(j < cnt ? li[j] : kTcNoId);
             }
         }
