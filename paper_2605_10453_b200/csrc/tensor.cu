@@ -20,7 +20,8 @@ namespace slimspec {
 static constexpr int kTcRows = 128;          // rows per tile = MMA M
 static constexpr int kTcKChunk = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
 static constexpr int kTcThreads = 192;
-static constexpr int kTcMaxK = 32;           // top-k entries a row keeps
+static constexpr int kTcMaxK = 32;           // largest k
+static constexpr int kTcList = 48;           // candidates a row parks before the list is compacted
 static constexpr int kTcNoId = 0x7fffffff;
 static constexpr float kLog2e = 1.4426950408889634f;
 
@@ -42,22 +43,26 @@ struct alignas(64) TcParams {
     int* err;
 };
 
-// Insert (value, id) into a row's list of the k best (values descending; of equal values the
-// earlier, lower id stays in front).  Returns the new threshold a candidate has to beat: the k-th
-// value once the list is full, else the row's starting bound thr0.
-__device__ __forceinline__ float topk_insert(float* lv, int* li, int& cnt, int k, float val, int id, float thr0)
+// A row's candidate list: up to kTcList (value, id) pairs above the row's threshold, appended in
+// the order the columns arrive (ascending id).  topk_compact sorts the list (values descending,
+// equal values keep their order, i.e. lower id first), cuts it to the k best and returns the
+// new threshold: the k-th value if the list holds k entries, else the old bound.
+__device__ __noinline__ float topk_compact(float* cv, int* ci, int& cnt, int k, float thr0)
 {
-    int pos = cnt < k ? cnt : k - 1;
-    if (cnt == k && !(val > lv[k - 1])) return lv[k - 1];
-    while (pos > 0 && lv[pos - 1] < val) {
-        lv[pos] = lv[pos - 1];
-        li[pos] = li[pos - 1];
-        --pos;
+    for (int i = 1; i < cnt; ++i) {
+        const float v = cv[i];
+        const int id = ci[i];
+        int pos = i;
+        while (pos > 0 && cv[pos - 1] < v) {
+            cv[pos] = cv[pos - 1];
+            ci[pos] = ci[pos - 1];
+            --pos;
+        }
+        cv[pos] = v;
+        ci[pos] = id;
     }
-    lv[pos] = val;
-    li[pos] = id;
-    cnt = cnt < k ? cnt + 1 : k;
-    return cnt == k ? lv[k - 1] : thr0;
+    if (cnt > k) cnt = k;
+    return cnt == k ? cv[k - 1] : thr0;
 }
 
 __device__ __forceinline__ float ex2_fast(float x)
@@ -166,8 +171,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         const bool live = m < p.M;
         const int k = p.k;
         float run_max = -FLT_MAX, run_sum = 0.f;
-        float lv[kTcMaxK];
-        int li[kTcMaxK];
+        float cv[kTcList];
+        int ci[kTcList];
         int cnt = 0;
         // Candidates must beat thr: the k-th best value once the list is full, before that a bound
         // known to lie below the row's k-th largest logit (from a sample of the vocabulary).
@@ -234,30 +239,25 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 for (int e = 0; e < 32; ++e) sacc[e & 3] += ex2_fast(fmaf(x[e], kLog2e, -mb));
                 run_sum += (sacc[0] + sacc[1]) + (sacc[2] + sacc[3]);
                 // top-k: ids arrive in ascending order, so a candidate must beat the threshold strictly.
-                // Only groups of eight whose maximum passes are looked at; what passes is parked and
-                // inserted after the scan, so the scan itself is compare-and-branch only.
+                // Only groups of eight whose maximum passes are looked at, and a candidate is merely
+                // appended; the list is sorted and cut when it overflows and once at the end.
                 if (cmax > thr) {
-                    float pend_v[8];
-                    int pend_i[8];
-                    int np = 0;
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         if (m8[q] > thr) {
 #pragma unroll
                             for (int e = 0; e < 8; ++e) {
                                 if (x[q * 8 + e] > thr) {
-                                    if (np == 8) {       // rare: flush the parked candidates
-                                        for (int j = 0; j < 8; ++j) thr = topk_insert(lv, li, cnt, k, pend_v[j], pend_i[j], thr0);
-                                        np = 0;
+                                    if (cnt == kTcList) thr = topk_compact(cv, ci, cnt, k, thr);
+                                    if (x[q * 8 + e] > thr) {
+                                        cv[cnt] = x[q * 8 + e];
+                                        ci[cnt] = col0 + q * 8 + e;
+                                        ++cnt;
                                     }
-                                    pend_v[np] = x[q * 8 + e];
-                                    pend_i[np] = col0 + q * 8 + e;
-                                    ++np;
                                 }
                             }
                         }
                     }
-                    for (int j = 0; j < np; ++j) thr = topk_insert(lv, li, cnt, k, pend_v[j], pend_i[j], thr0);
                 }
             }
             if (p.mode == 3 && live) p.smax[(size_t)ct * p.nrb * kTcRows + m] = f2key(tile_max);
@@ -265,12 +265,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             mbar_arrive(&acc_empty[buf]);
         }
         if (alive && live && p.mode == 0) {
+            topk_compact(cv, ci, cnt, k, thr);
             float* rec = p.part + ((size_t)m * p.gct + cg) * p.rec_words;
             rec[0] = run_max;
             rec[1] = run_sum;
             for (int j = 0; j < k; ++j) {
-                rec[2 + j] = __uint_as_float(j < cnt ? f2key(lv[j] + 0.f) : 0u);      // -0 and +0 rank alike
-                rec[2 + k + j] = __int_as_float(j < cnt ? li[j] : kTcNoId);
+                rec[2 + j] = __uint_as_float(j < cnt ? f2key(cv[j] + 0.f) : 0u);      // -0 and +0 rank alike
+                rec[2 + k + j] = __int_as_float(j < cnt ? ci[j] : kTcNoId);
             }
         }
     }
