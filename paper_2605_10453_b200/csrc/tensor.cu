@@ -38,6 +38,8 @@ struct alignas(64) TcParams {
     const uint32_t* thr0;   // mode 0: per-row lower bound (key - 1) of the k-th largest logit, or null
     int k;
     int rec_words;
+    int ns;                 // ring stages
+    int xres;               // 1: the row block's whole X (K <= 512) is loaded once and stays in shared memory
     float* out;
     float* part;            // records [M][gct][rec_words]
     int* err;
@@ -76,20 +78,25 @@ __device__ __forceinline__ float ex2_fast(float x)
 template <int NV>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant__ TcParams p)
 {
-    constexpr int NS = (NV == 256) ? 4 : 6;                 // ring stages
+    constexpr int NSMAX = 8;                                // most ring stages
     constexpr int X_BYTES = kTcRows * kTcKChunk * 2;        // 16 KB
     constexpr int WBOX_BYTES = kTcKChunk * 64 * 2;          // 8 KB: 64 k x 64 columns
     constexpr int W_BYTES = WBOX_BYTES * (NV / 64);
-    constexpr int STAGE = X_BYTES + W_BYTES;
+    const int NS = p.ns;
+    const bool xres = p.xres != 0;
+    // a stage holds a W chunk, and an X chunk in front of it unless X is resident
+    const int STAGE = xres ? W_BYTES : X_BYTES + W_BYTES;
+    const int W_OFF = xres ? 0 : X_BYTES;
     // instruction descriptor: D fp32, A and B bf16, A K-major, B MN-major, N = NV, M = 128
     constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                ((uint32_t)(NV >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
 
     extern __shared__ unsigned char smem_raw[];
-    __shared__ uint64_t full[NS], empty[NS], acc_full[2], acc_empty[2];
+    __shared__ uint64_t full[NSMAX], empty[NSMAX], acc_full[2], acc_empty[2], x_full;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    unsigned char* stages = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char* xarea = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char* stages = xarea + (xres ? (size_t)p.chunks_per_split * X_BYTES : 0);
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -104,6 +111,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+        mbar_init(&x_full, 1);
         abort_s = 0;
         mbar_fence_init();
         prefetch_tensor_map(&p.mapX);
@@ -120,18 +128,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         if (lane == 0) {
             int it = 0;
             bool alive = true;
+            if (xres && ntiles > 0) {
+                mbar_arrive_expect_tx(&x_full, (uint32_t)cps * X_BYTES);
+                for (int c = 0; c < cps; ++c)
+                    tma_load_2d(xarea + (size_t)c * X_BYTES, &p.mapX, c * kTcKChunk, rb * kTcRows, &x_full);
+            }
             for (int t = 0; t < ntiles && alive; ++t) {
                 const int ct = cg + t * p.gct;
                 for (int c = 0; c < cps; ++c, ++it) {
                     const int s = it % NS, use = it / NS;
                     if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, p.err, ERR_WAIT_EMPTY)) { alive = false; break; }
                     unsigned char* st = stages + (size_t)s * STAGE;
-                    mbar_arrive_expect_tx(&full[s], STAGE);
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)STAGE);
                     const int kx = (ks * cps + c) * kTcKChunk;
-                    tma_load_2d(st, &p.mapX, kx, rb * kTcRows, &full[s]);
+                    if (!xres) tma_load_2d(st, &p.mapX, kx, rb * kTcRows, &full[s]);
 #pragma unroll
                     for (int i = 0; i < NV / 64; ++i)
-                        tma_load_2d(st + X_BYTES + i * WBOX_BYTES, &p.mapW, ct * NV + i * 64, kx, &full[s]);
+                        tma_load_2d(st + W_OFF + i * WBOX_BYTES, &p.mapW, ct * NV + i * 64, kx, &full[s]);
                 }
             }
         }
@@ -140,6 +153,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         if (lane == 0) {
             int it = 0;
             bool alive = true;
+            if (xres && ntiles > 0 && !mbar_wait(&x_full, 0, abort_flag, p.err, ERR_WAIT_FULL)) alive = false;
             for (int t = 0; t < ntiles && alive; ++t) {
                 const int buf = t & 1;
                 if (t >= 2 && !mbar_wait(&acc_empty[buf], ((t >> 1) - 1) & 1, abort_flag, p.err, ERR_WAIT_FREE)) break;
@@ -149,9 +163,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                     const int s = it % NS, use = it / NS;
                     if (!mbar_wait(&full[s], use & 1, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t xa = smem_u32(stages + (size_t)s * STAGE);
+                    const uint32_t sa = smem_u32(stages + (size_t)s * STAGE);
+                    const uint32_t xa = xres ? smem_u32(xarea + (size_t)c * X_BYTES) : sa;
                     const uint64_t a_desc = tc_smem_desc_sw128(xa, 16, 1024);
-                    const uint64_t b_desc = tc_smem_desc_sw128(xa + X_BYTES, WBOX_BYTES, 1024);
+                    const uint64_t b_desc = tc_smem_desc_sw128(sa + W_OFF, WBOX_BYTES, 1024);
 #pragma unroll
                     for (int j = 0; j < kTcKChunk / 16; ++j) {
                         // 16 of K per instruction: 32 bytes along a K-major row, two 8-row groups of the N-major tile
@@ -239,19 +254,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 for (int e = 0; e < 32; ++e) sacc[e & 3] += ex2_fast(fmaf(x[e], kLog2e, -mb));
                 run_sum += (sacc[0] + sacc[1]) + (sacc[2] + sacc[3]);
                 // top-k: ids arrive in ascending order, so a candidate must beat the threshold strictly.
-                // Only groups of eight whose maximum passes are looked at, and a candidate is merely
-                // appended; the list is sorted and cut when it overflows and once at the end.
-                if (cmax > thr) {
+                // Some row of the warp has a candidate in most chunks, but a given row rarely has
+                // one and hardly ever two.  So a lane with a candidate builds the bit mask of its
+                // columns above its threshold with straight-line code; a single set bit is the chunk
+                // maximum and is appended without indexing registers; only two or more take the
+                // branchy scan.
+                if (cmax > thr) {      // no warp-wide vote here: lanes of rows past M have left the loop body
+                    uint32_t gt = 0u;
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        if (m8[q] > thr) {
+                    for (int e = 0; e < 32; ++e) gt |= (x[e] > thr) ? (1u << e) : 0u;
+                    if (gt != 0u) {
+                        if ((gt & (gt - 1u)) == 0u) {
+                            if (cnt == kTcList) thr = topk_compact(cv, ci, cnt, k, thr);
+                            cv[cnt] = cmax;
+                            ci[cnt] = col0 + __ffs(gt) - 1;
+                            ++cnt;
+                        } else {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                if (x[q * 8 + e] > thr) {
+                            for (int e = 0; e < 32; ++e) {
+                                if (x[e] > thr) {
                                     if (cnt == kTcList) thr = topk_compact(cv, ci, cnt, k, thr);
-                                    if (x[q * 8 + e] > thr) {
-                                        cv[cnt] = x[q * 8 + e];
-                                        ci[cnt] = col0 + q * 8 + e;
+                                    if (x[e] > thr) {
+                                        cv[cnt] = x[e];
+                                        ci[cnt] = col0 + e;
                                         ++cnt;
                                     }
                                 }
@@ -421,12 +446,22 @@ bool tensor_ok(int M, int K, int N, int k, int mode)
     return true;
 }
 
+static constexpr size_t kTcSmemMax = 227 * 1024;
+
+// Chooses the ring depth (and whether X can stay resident) and launches.
 template <int NV>
-static cudaError_t launch_gemm(const TcParams& p, int grid, cudaStream_t st)
+static cudaError_t launch_gemm(TcParams p, int grid, cudaStream_t st)
 {
-    constexpr int NS = (NV == 256) ? 4 : 6;
-    constexpr int STAGE = kTcRows * kTcKChunk * 2 + kTcKChunk * NV * 2;
-    const size_t smem = (size_t)NS * STAGE + 1024;
+    const size_t x_bytes = (size_t)kTcRows * kTcKChunk * 2, w_bytes = (size_t)kTcKChunk * NV * 2;
+    const size_t x_all = (size_t)p.chunks_per_split * x_bytes;
+    p.xres = (p.nks == 1 && x_all + 3 * w_bytes + 1024 <= kTcSmemMax) ? 1 : 0;
+    const size_t stage = p.xres ? w_bytes : x_bytes + w_bytes;
+    const size_t fixed = 1024 + (p.xres ? x_all : 0);
+    int ns = (int)((kTcSmemMax - fixed) / stage);
+    if (ns > 8) ns = 8;
+    if (ns < 2) return cudaErrorInvalidValue;
+    p.ns = ns;
+    const size_t smem = fixed + (size_t)ns * stage;
     auto kern = k_tc_gemm<NV>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
