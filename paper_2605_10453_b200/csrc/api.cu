@@ -71,7 +71,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     // tensor path 128 * nrb rows x (SMs / nrb) slabs
     const int rec_k = max_k < 32 ? max_k : 32;
     const size_t mpad128 = (size_t)round_up(max_M, 128);
-    const size_t part_elems = ((size_t)kRowPad * 256 + (size_t)(c->sm_count + 8) * 128 + mpad128) *
+    const size_t part_elems = ((size_t)kRowPad * 256 + (size_t)(c->sm_count + 12) * 256 + 2 * mpad128) *
                               (size_t)round_up(2 + 2 * rec_k, 4);
     // K-split partial tiles of the tensor-core down-projection: one 128 x 128 fp32 tile per SM, or one split
     size_t zpart_elems = (size_t)(c->sm_count + 12) * 128 * 128;

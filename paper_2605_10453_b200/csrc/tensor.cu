@@ -5,10 +5,10 @@
 //   full-rank head   logits = h W X = h, W = W, same epilogue
 // (Section 4.1; the softmax of Section 3.2 and the candidate selection.)
 //
-// One CTA per SM, six warps: warp 0 feeds a ring of shared-memory stages by TMA, one thread of
+// One CTA per SM, ten warps: warp 0 feeds a ring of shared-memory stages by TMA, one thread of
 // warp 1 issues the MMAs (128 rows x NV columns x 16 per instruction) into one of two
-// accumulator buffers in tensor memory, warps 2-5 read the finished buffer (a thread per row) and
-// keep that row's running max / sum-exp / top-k while the next tile's MMAs run.
+// accumulator buffers in tensor memory, warps 2-9 read the finished buffer (a thread per row and
+// column half) and keep that row's running max / sum-exp / top-k while the next tile's MMAs run.
 #include "kernels.h"
 #include "ptx.cuh"
 #include <cuda.h>
@@ -19,7 +19,7 @@ namespace slimspec {
 
 static constexpr int kTcRows = 128;          // rows per tile = MMA M
 static constexpr int kTcKChunk = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
-static constexpr int kTcThreads = 192;
+static constexpr int kTcThreads = 320;       // TMA warp, MMA warp, eight epilogue warps
 static constexpr int kTcMaxK = 32;           // largest k
 static constexpr int kTcList = 48;           // candidates a row parks before the list is compacted
 static constexpr int kTcNoId = 0x7fffffff;
@@ -41,7 +41,7 @@ struct alignas(64) TcParams {
     int ns;                 // ring stages
     int xres;               // 1: the row block's whole X (K <= 512) is loaded once and stays in shared memory
     float* out;
-    float* part;            // records [M][gct][rec_words]
+    float* part;            // records [M][2 * gct][rec_words]: two column halves per CTA
     int* err;
 };
 
@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 128); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 256); }
         mbar_init(&x_full, 1);
         abort_s = 0;
         mbar_fence_init();
@@ -181,6 +181,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
     } else {
         // ================= epilogue: thread = row =================
         const int quarter = warp & 3;                        // the lane quarter this warp may read
+        const int half = (warp - 2) >> 2;                    // two warps share a quarter: each takes half the columns
         const int row = quarter * 32 + lane;
         const int m = rb * kTcRows + row;
         const bool live = m < p.M;
@@ -203,7 +204,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NV);
             float tile_max = -FLT_MAX;
 #pragma unroll 1
-            for (int c0 = 0; c0 < NV; c0 += 32) {
+            for (int c0 = half * (NV / 2); c0 < (half + 1) * (NV / 2); c0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32x32(taddr + (uint32_t)c0, v);
                 tmem_ld_wait();
@@ -285,13 +286,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                     }
                 }
             }
-            if (p.mode == 3 && live) p.smax[(size_t)ct * p.nrb * kTcRows + m] = f2key(tile_max);
+            if (p.mode == 3 && live) p.smax[((size_t)ct * 2 + half) * p.nrb * kTcRows + m] = f2key(tile_max);
             tc_fence_before_sync();
             mbar_arrive(&acc_empty[buf]);
         }
         if (alive && live && p.mode == 0) {
             topk_compact(cv, ci, cnt, k, thr);
-            float* rec = p.part + ((size_t)m * p.gct + cg) * p.rec_words;
+            float* rec = p.part + ((size_t)m * (2 * p.gct) + 2 * cg + half) * p.rec_words;
             rec[0] = run_max;
             rec[1] = run_sum;
             for (int j = 0; j < k; ++j) {
@@ -347,7 +348,7 @@ __global__ void __launch_bounds__(256) k_tc_thr0(const uint32_t* __restrict__ sm
 }
 
 // ------------------------------------------------------------------------------------------
-// Merge the P per-slab records of each row: one warp per row, a lane owns up to 8 slab lists.
+// Merge the P per-slab records of each row: one warp per row, a lane owns up to 10 slab lists.
 __global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part, int M, int P, int RW, int k,
                                                   int32_t* __restrict__ ids, float* __restrict__ logprobs)
 {
@@ -363,10 +364,10 @@ __global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part
         gs += __ldcg(rows + (size_t)s * RW + 1) * __expf(__ldcg(rows + (size_t)s * RW) - gm);
     gs = warp_sum(gs);
     const float lse = gm + __logf(gs);
-    uint32_t hk[8];
-    int hi[8], hp[8];
+    uint32_t hk[10];
+    int hi[10], hp[10];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
+    for (int q = 0; q < 10; ++q) {
         const int s = lane + 32 * q;
         hp[q] = 0;
         hk[q] = (s < P) ? __float_as_uint(__ldcg(rows + (size_t)s * RW + 2)) : 0u;
@@ -378,7 +379,7 @@ __global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part
         uint32_t bk = hk[0];
         int bi = hi[0], bs = 0;
 #pragma unroll
-        for (int q = 1; q < 8; ++q) {
+        for (int q = 1; q < 10; ++q) {
             const bool better = hk[q] > bk || (hk[q] == bk && hi[q] < bi);
             bk = better ? hk[q] : bk;
             bi = better ? hi[q] : bi;
@@ -389,7 +390,7 @@ __global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part
         const bool win = (bk == wk) && ((uint32_t)bi == wi);
         if (win && wk != 0u) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
+            for (int q = 0; q < 10; ++q) {
                 if (q == bs) {
                     const int s = lane + 32 * q;
                     const int np = hp[q] + 1;
@@ -487,21 +488,22 @@ cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k
     p.gct = sm_count / p.nrb;
     if (p.gct < 1) p.gct = 1;
     if (p.gct > p.nct) p.gct = p.nct;
-    if (p.gct > 256) p.gct = 256;
+    if (p.gct > 160) p.gct = 160;       // the merge takes up to 320 lists per row
     p.mode = mode;
     p.k = k;
     p.rec_words = (2 + 2 * k + 3) / 4 * 4;
     p.out = logits;
     p.part = s.part;
     p.err = s.err;
-    if (mode == 0 && (size_t)M * p.gct * p.rec_words > s.part_elems) return cudaErrorInvalidValue;
+    if (mode == 0 && (size_t)M * 2 * p.gct * p.rec_words > s.part_elems) return cudaErrorInvalidValue;
     cudaError_t e;
     if (mode == 0) {
         // A bound below each row's k-th largest logit, from the first sample tiles of the vocabulary:
         // it keeps the per-row candidate lists of the main pass almost idle.
-        int nst = 2 * k > 32 ? 2 * k : 32;
+        // (each sample tile yields two maxima per row, one per column half; k_tc_thr0 takes up to 64)
+        int nst = k > 16 ? 32 : 16;
         if (nst > p.nct) nst = p.nct;
-        if (nst >= k && (size_t)nst * p.nrb * kTcRows <= s.smax_elems) {
+        if (2 * nst >= k && (size_t)2 * nst * p.nrb * kTcRows <= s.smax_elems) {
             TcParams q = p;
             q.mode = 3;
             q.nct = nst;
@@ -509,7 +511,7 @@ cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k
             q.smax = s.smax;
             e = (nv == 128) ? launch_gemm<128>(q, nst * p.nrb, st) : launch_gemm<256>(q, nst * p.nrb, st);
             if (e != cudaSuccess) return e;
-            k_tc_thr0<<<(M + 7) / 8, 256, 0, st>>>(s.smax, nst, p.nrb * kTcRows, M, k, s.thr0);
+            k_tc_thr0<<<(M + 7) / 8, 256, 0, st>>>(s.smax, 2 * nst, p.nrb * kTcRows, M, k, s.thr0);
             e = cudaGetLastError();
             if (e != cudaSuccess) return e;
             *launches += 2;
@@ -521,7 +523,7 @@ cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k
     if (e != cudaSuccess) return e;
     *launches += 1;
     if (mode == 0) {
-        k_tc_merge<<<(M + 7) / 8, 256, 0, st>>>(s.part, M, p.gct, p.rec_words, k, ids, logprobs);
+        k_tc_merge<<<(M + 7) / 8, 256, 0, st>>>(s.part, M, 2 * p.gct, p.rec_words, k, ids, logprobs);
         *launches += 1;
         e = cudaGetLastError();
     }
