@@ -29,7 +29,8 @@ struct slimspec_ctx {
 static const int kTimingEvents = 256;
 
 static const int kMaxParts = 256;      // most V slabs any kernel writes per row
-static const int kStreamMaxRows = 8;   // largest M the streaming path is chosen for
+static const int kStreamMaxRows = 4;   // largest M the streaming path is chosen for
+static const int kFmaDownprojRows = 0;  // tensor path: down-projection by FMAs up to this many rows
 static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
@@ -258,13 +259,16 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         int n = 0;
         const bf16* X = h;
         if (lowrank) {
-            cudaError_t e0 = tensor_downproj(h, A, M, d, r, c->s, c->sm_count, &n, st);
+            // few rows: the FMA kernel (one launch) beats a K-split tensor-core GEMM plus its reduction
+            cudaError_t e0;
+            if (M <= kFmaDownprojRows && r % 16 == 0) { e0 = stream_downproj_bf16(h, A, M, d, r, c->s.zb, st); n = 1; }
+            else e0 = tensor_downproj(h, A, M, d, r, c->s, c->sm_count, &n, st);
             c->launches += n;
             n = 0;
             if (e0 != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
             X = c->s.zb;
         }
-        cudaError_t e = tensor_head(X, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, &n, st);
+        cudaError_t e = tensor_head(X, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, lowrank, &n, st);
         c->launches += n;
         if (e != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         return SLIMSPEC_OK;

@@ -47,6 +47,8 @@ StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count);
 // z^T = (h A)^T for M <= 8 rows, rows M..mt-1 zero-filled; r must be a multiple of 16.
 cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
                             cudaStream_t st);
+// z (bf16 [M][r]) = h A with FP32 FMAs, any M (A is re-read once per eight rows); r a multiple of 16.
+cudaError_t stream_downproj_bf16(const bf16* h, const bf16* A, int M, int d, int r, bf16* zb, cudaStream_t st);
 // z^T = widened h^T (full-rank head: no down-projection).
 cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st);
 // logits = z B streamed once; mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
@@ -61,7 +63,10 @@ bool tensor_ok(int M, int K, int N, int k, int mode);
 cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, const Scratch& s, int sm_count,
                             int* launches, cudaStream_t st);
 // X W with X bf16 [M][K], W bf16 [K][N]; mode 0: fused log-softmax / top-k, mode 1: raw fp32 logits.
+// after_kernel: X is written by the kernel launched just before on `st` (the first kernel here is
+// then launched as its programmatic dependent).
 cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
-                        float* logprobs, float* logits, const Scratch& s, int sm_count, int* launches, cudaStream_t st);
+                        float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
+                        cudaStream_t st);
 
 }  // namespace slimspec

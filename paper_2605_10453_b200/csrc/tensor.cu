@@ -122,6 +122,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_s;
+    // Everything above touched no global data: under programmatic dependent launch it overlaps the
+    // kernel before; from here on that kernel's results are needed.
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 0) {
         // ================= producer: one thread issues the TMA loads =================
@@ -312,6 +316,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
 // z = sum of the K-split partial tiles, rounded once to bf16.
 __global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad, int M, int r, bf16* __restrict__ z)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= M * r) return;
     const int m = e / r, j = e - m * r;
@@ -333,6 +339,8 @@ __global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad,
 __global__ void __launch_bounds__(256) k_tc_thr0(const uint32_t* __restrict__ smax, int nst, int mpad, int M, int k,
                                                  uint32_t* __restrict__ thr0)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m = blockIdx.x * (blockDim.x >> 5) + warp;
     if (m >= M) return;
@@ -348,38 +356,51 @@ __global__ void __launch_bounds__(256) k_tc_thr0(const uint32_t* __restrict__ sm
 }
 
 // ------------------------------------------------------------------------------------------
-// Merge the P per-slab records of each row: one warp per row, a lane owns up to 10 slab lists.
-__global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part, int M, int P, int RW, int k,
+// Merge the P per-slab records of each row: one warp per row, a lane owns up to 10 slab lists
+// and keeps each list's head and the entry after it in registers, so that a pop never waits for
+// memory unless the same list wins twice in a row.
+static constexpr int kMergeLists = 10;
+
+__global__ void __launch_bounds__(128) k_tc_merge(const float* __restrict__ part, int M, int P, int RW, int k,
                                                   int32_t* __restrict__ ids, float* __restrict__ logprobs)
 {
+    pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m = blockIdx.x * (blockDim.x >> 5) + warp;
     if (m >= M) return;
     const float* rows = part + (size_t)m * P * RW;
+    uint32_t hk[kMergeLists], nk[kMergeLists];
+    int hi[kMergeLists], ni[kMergeLists], hp[kMergeLists];
+    float pm[kMergeLists], ps[kMergeLists];
+#pragma unroll
+    for (int q = 0; q < kMergeLists; ++q) {
+        const int s = lane + 32 * q;
+        const bool have = s < P;
+        const float* rec = rows + (size_t)(have ? s : 0) * RW;
+        hp[q] = 0;
+        pm[q] = have ? __ldcg(rec) : -FLT_MAX;
+        ps[q] = have ? __ldcg(rec + 1) : 0.f;
+        hk[q] = have ? __float_as_uint(__ldcg(rec + 2)) : 0u;
+        hi[q] = have ? __float_as_int(__ldcg(rec + 2 + k)) : kTcNoId;
+        nk[q] = (have && k > 1) ? __float_as_uint(__ldcg(rec + 3)) : 0u;
+        ni[q] = (have && k > 1) ? __float_as_int(__ldcg(rec + 3 + k)) : kTcNoId;
+    }
     float gm = -FLT_MAX;
-    for (int s = lane; s < P; s += 32) gm = fmaxf(gm, __ldcg(rows + (size_t)s * RW));
+#pragma unroll
+    for (int q = 0; q < kMergeLists; ++q) gm = fmaxf(gm, pm[q]);
     gm = warp_max(gm);
     float gs = 0.f;
-    for (int s = lane; s < P; s += 32)
-        gs += __ldcg(rows + (size_t)s * RW + 1) * __expf(__ldcg(rows + (size_t)s * RW) - gm);
+#pragma unroll
+    for (int q = 0; q < kMergeLists; ++q) gs += ps[q] * __expf(pm[q] - gm);
     gs = warp_sum(gs);
     const float lse = gm + __logf(gs);
-    uint32_t hk[10];
-    int hi[10], hp[10];
-#pragma unroll
-    for (int q = 0; q < 10; ++q) {
-        const int s = lane + 32 * q;
-        hp[q] = 0;
-        hk[q] = (s < P) ? __float_as_uint(__ldcg(rows + (size_t)s * RW + 2)) : 0u;
-        hi[q] = (s < P) ? __float_as_int(__ldcg(rows + (size_t)s * RW + 2 + k)) : kTcNoId;
-    }
     uint32_t ok = 0;
     int oi = kTcNoId;
     for (int j = 0; j < k; ++j) {
         uint32_t bk = hk[0];
         int bi = hi[0], bs = 0;
 #pragma unroll
-        for (int q = 1; q < 10; ++q) {
+        for (int q = 1; q < kMergeLists; ++q) {
             const bool better = hk[q] > bk || (hk[q] == bk && hi[q] < bi);
             bk = better ? hk[q] : bk;
             bi = better ? hi[q] : bi;
@@ -387,17 +408,19 @@ __global__ void __launch_bounds__(256) k_tc_merge(const float* __restrict__ part
         }
         const uint32_t wk = warp_max_u32(bk);
         const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
-        const bool win = (bk == wk) && ((uint32_t)bi == wi);
-        if (win && wk != 0u) {
+        const bool win = (bk == wk) && ((uint32_t)bi == wi) && wk != 0u;
 #pragma unroll
-            for (int q = 0; q < 10; ++q) {
-                if (q == bs) {
-                    const int s = lane + 32 * q;
-                    const int np = hp[q] + 1;
-                    hp[q] = np;
-                    hk[q] = (np < k) ? __float_as_uint(__ldcg(rows + (size_t)s * RW + 2 + np)) : 0u;
-                    hi[q] = (np < k) ? __float_as_int(__ldcg(rows + (size_t)s * RW + 2 + k + np)) : kTcNoId;
-                }
+        for (int q = 0; q < kMergeLists; ++q) {
+            if (win && q == bs) {
+                const int s = lane + 32 * q;
+                const int np = hp[q] + 1;
+                hp[q] = np;
+                hk[q] = nk[q];
+                hi[q] = ni[q];
+                const bool more = np + 1 < k;
+                const float* rec = rows + (size_t)s * RW;
+                nk[q] = more ? __float_as_uint(__ldcg(rec + 3 + np)) : 0u;
+                ni[q] = more ? __float_as_int(__ldcg(rec + 3 + k + np)) : kTcNoId;
             }
         }
         if (lane == j) { ok = wk; oi = (int)wi; }
@@ -449,9 +472,28 @@ bool tensor_ok(int M, int K, int N, int k, int mode)
 
 static constexpr size_t kTcSmemMax = 227 * 1024;
 
+// Launch with (or without) the programmatic-dependent-launch attribute: the kernel may start while
+// the one before it in the stream is still running and meets it at griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_chain(void (*kern)(KArgs...), int grid, int block, size_t smem, bool pdl, cudaStream_t st,
+                                Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 // Chooses the ring depth (and whether X can stay resident) and launches.
 template <int NV>
-static cudaError_t launch_gemm(TcParams p, int grid, cudaStream_t st)
+static cudaError_t launch_gemm(TcParams p, int grid, bool pdl, cudaStream_t st)
 {
     const size_t x_bytes = (size_t)kTcRows * kTcKChunk * 2, w_bytes = (size_t)kTcKChunk * NV * 2;
     const size_t x_all = (size_t)p.chunks_per_split * x_bytes;
@@ -466,14 +508,14 @@ static cudaError_t launch_gemm(TcParams p, int grid, cudaStream_t st)
     auto kern = k_tc_gemm<NV>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kTcThreads, smem, st>>>(p);
-    return cudaGetLastError();
+    return launch_chain(kern, grid, kTcThreads, smem, pdl, st, p);
 }
 
 // out = X W through the tensor cores.  mode 0: top-k records then merge into ids / logprobs;
 // mode 1: fp32 logits.  X is bf16 [M][K], W bf16 [K][N].
 cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
-                        float* logprobs, float* logits, const Scratch& s, int sm_count, int* launches, cudaStream_t st)
+                        float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
+                        cudaStream_t st)
 {
     TcParams p;
     memset(&p, 0, sizeof(p));
@@ -509,23 +551,24 @@ cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k
             q.nct = nst;
             q.gct = nst;
             q.smax = s.smax;
-            e = (nv == 128) ? launch_gemm<128>(q, nst * p.nrb, st) : launch_gemm<256>(q, nst * p.nrb, st);
+            e = (nv == 128) ? launch_gemm<128>(q, nst * p.nrb, after_kernel, st) : launch_gemm<256>(q, nst * p.nrb, after_kernel, st);
             if (e != cudaSuccess) return e;
-            k_tc_thr0<<<(M + 7) / 8, 256, 0, st>>>(s.smax, 2 * nst, p.nrb * kTcRows, M, k, s.thr0);
-            e = cudaGetLastError();
+            e = launch_chain(k_tc_thr0, (M + 7) / 8, 256, 0, true, st, (const uint32_t*)s.smax, 2 * nst, p.nrb * kTcRows, M, k,
+                             s.thr0);
+            after_kernel = true;
             if (e != cudaSuccess) return e;
             *launches += 2;
             p.thr0 = s.thr0;
         }
     }
     const int grid = p.gct * p.nrb;
-    e = (nv == 128) ? launch_gemm<128>(p, grid, st) : launch_gemm<256>(p, grid, st);
+    e = (nv == 128) ? launch_gemm<128>(p, grid, after_kernel, st) : launch_gemm<256>(p, grid, after_kernel, st);
     if (e != cudaSuccess) return e;
     *launches += 1;
     if (mode == 0) {
-        k_tc_merge<<<(M + 7) / 8, 256, 0, st>>>(s.part, M, 2 * p.gct, p.rec_words, k, ids, logprobs);
+        e = launch_chain(k_tc_merge, (M + 3) / 4, 128, 0, true, st, (const float*)s.part, M, 2 * p.gct, p.rec_words, k, ids,
+                         logprobs);
         *launches += 1;
-        e = cudaGetLastError();
     }
     return e;
 }
@@ -555,12 +598,13 @@ cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, c
     p.err = s.err;
     const size_t need = (size_t)nks * p.nrb * kTcRows * r;
     if (need > s.zpart_elems) return cudaErrorInvalidValue;
-    cudaError_t e = launch_gemm<128>(p, p.nrb * p.nct * nks, st);
+    cudaError_t e = launch_gemm<128>(p, p.nrb * p.nct * nks, false, st);
     if (e != cudaSuccess) return e;
     const int n = M * r;
-    k_tc_reduce_z<<<(n + 255) / 256, 256, 0, st>>>(s.zpart, nks, p.nrb * kTcRows, M, r, s.zb);
+    e = launch_chain(k_tc_reduce_z, (n + 255) / 256, 256, 0, true, st, (const float*)s.zpart, nks, p.nrb * kTcRows, M, r,
+                     s.zb);
     *launches += 2;
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace slimspec
