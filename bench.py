@@ -2,6 +2,7 @@
 """Benchmark of the draft LM-head forward (low-rank head, fused log-softmax / top-k).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extra]
+    python bench.py --sweep        (d=8192 rank / batch sweep: one line per point, then a table)
 
 One step = one call of slimspec_head_topk: down-projection, the streamed up-projection,
 online log-softmax, top-k and the slab merge, on the 8B-class head at M = 1
@@ -360,6 +361,70 @@ def extra_points(torch, ctx, synth, binding, dev, peaks):
     return out
 
 
+def run_sweep(args):
+    """The rank / batch sweep (d=8192, V=128256, r in {d/16, d/8, d/4} and full rank, M in {1..1024}):
+    one JSON line per point with us/call and the fraction of the roofline, then a markdown table.
+    Weights are drawn on the device from a seeded generator (values do not change the timing)."""
+    import torch
+    from paper_2605_10453_b200 import binding, build, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    build.build()
+    peaks, kind = load_peaks()
+    d, V, k = synth.SWEEP_D, synth.SWEEP_V, 10
+    ctx = binding.Context(max_M=max(synth.SWEEP_MS), max_d=d, max_V=V, max_k=16)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+
+    def draw(rows, cols, std):
+        return (torch.randn((rows, cols), generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+
+    rows_out = []
+    for r in list(synth.SWEEP_RANKS) + [0]:
+        full = r == 0
+        nbytes = 2 * d * V if full else 2 * (d * r + r * V)
+        R = max(1, min(4, -(-2 * L2_BYTES // nbytes)))
+        if full:
+            Ws = [draw(d, V, d ** -0.5) for _ in range(R)]
+        else:
+            As = [draw(d, r, d ** -0.5) for _ in range(R)]
+            Bs = [draw(r, V, r ** -0.5) for _ in range(R)]
+        for M in synth.SWEEP_MS:
+            h = draw(M, d, 1.0)
+            ids = torch.empty((M, k), dtype=torch.int32, device=dev)
+            lp = torch.empty((M, k), dtype=torch.float32, device=dev)
+            if full:
+                fn = lambda i: ctx.fullhead_topk(h, Ws[i % R], k, out_ids=ids, out_logprobs=lp)
+                byt, flo = 2 * d * V + 2 * M * d, 2 * M * d * V
+            else:
+                fn = lambda i: ctx.slimspec_head_topk(h, As[i % R], Bs[i % R], k, out_ids=ids, out_logprobs=lp)
+                byt, flo = head_bytes(M, d, r, V, k), head_flops(M, d, r, V)
+            n = max(3, min(100, int(2e4 / (byt / (peaks["hbm_gbs"] * 1e3) + flo / (peaks["bf16_tflops"] * 1e6)))))
+            for i in range(3):
+                fn(i)
+            us = time_calls(torch, fn, n) * 1e3 / n
+            t_hbm, t_mma = byt / (peaks["hbm_gbs"] * 1e9) * 1e6, flo / (peaks["bf16_tflops"] * 1e12) * 1e6
+            roof = max(t_hbm, t_mma)
+            row = {"sweep": "c4", "rank": "full" if full else r, "M": M, "us_per_call": us, "roofline_us": roof,
+                   "roofline_frac": roof / us, "bound": "hbm" if t_hbm >= t_mma else "tensor", "peaks": kind,
+                   "path": {1: "generic", 2: "stream", 3: "tensor"}.get(ctx.last_path(), "?"), "calls": n}
+            if ctx.last_error() != binding.OK:
+                raise SystemExit("device-side wait timed out in the sweep")
+            rows_out.append(row)
+            print(json.dumps(row), flush=True)
+        if full:
+            del Ws
+        else:
+            del As, Bs
+        torch.cuda.empty_cache()
+    print("| rank | M | path | us/call | roofline us | fraction | bound |")
+    print("|---|---|---|---|---|---|---|")
+    for r_ in rows_out:
+        print("| %s | %d | %s | %.1f | %.1f | %.2f | %s |" % (r_["rank"], r_["M"], r_["path"], r_["us_per_call"],
+                                                          r_["roofline_us"], r_["roofline_frac"], r_["bound"]))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -367,8 +432,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the extra points and the CPU baseline")
+    ap.add_argument("--sweep", action="store_true", help="run the rank / batch sweep instead of the benchmark line")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

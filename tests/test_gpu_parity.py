@@ -197,6 +197,24 @@ def test_throughput_batch_sampled_rows(ctx):
         assert np.max(np.abs(l1.cpu().numpy()[0] - lp[m])) < 2e-4
 
 
+@pytest.mark.parametrize("r,M", [(1024, 64), (2048, 4)])
+def test_sweep_shapes_sampled_rows(r, M):
+    # d = 8192 heads of the rank sweep: K too long for a resident code / X, several z chunks
+    d, V, k = synth.SWEEP_D, synth.SWEEP_V, 10
+    c = binding.Context(max_M=M, max_d=d, max_V=V, max_k=16)
+    x = synth.make_inputs(M, d, r, V, seed=7)
+    g = dev(x)
+    ids, lp = c.slimspec_head_topk(g["h"], g["A"], g["B"], k)
+    torch.cuda.synchronize()
+    assert c.last_error() == binding.OK
+    rows = sorted({0, M // 2, M - 1})
+    b = obits(x)
+    ref = oracle.head_topk(b["h"][rows], b["A"], b["B"], k)
+    st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy(), rows=rows)
+    assert st["max_lp_err"] <= LOGPROB_TOL
+    c.close()
+
+
 # ---------------------------------------------------------------- full-rank baseline, logits
 
 @pytest.mark.parametrize("M", [1, 8])
