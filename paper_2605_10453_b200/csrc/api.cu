@@ -30,7 +30,7 @@ static const int kTimingEvents = 256;
 
 static const int kMaxParts = 256;      // most V slabs any kernel writes per row
 static const int kStreamMaxRows = 4;   // largest M the streaming path is chosen for
-static const int kFmaDownprojRows = 0;  // tensor path: down-projection by FMAs up to this many rows
+static const int kSplitCodeRows = 64;   // tensor path: z carried as hi + lo bf16 parts up to this many rows
 static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
@@ -81,7 +81,8 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     ok = ok && cudaMalloc(&c->s.z, z_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->s.zb, mpad128 * (size_t)max_d * sizeof(bf16)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.zb, 2 * mpad128 * (size_t)max_d * sizeof(bf16)) == cudaSuccess;
+    if (ok) c->s.zb_lo = c->s.zb + mpad128 * (size_t)max_d;
     ok = ok && cudaMalloc(&c->s.smax, 64 * mpad128 * sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.thr0, mpad128 * sizeof(uint32_t)) == cudaSuccess;
     c->s.smax_elems = 64 * mpad128;
@@ -258,17 +259,19 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
     if (path == SLIMSPEC_PATH_TENSOR) {
         int n = 0;
         const bf16* X = h;
+        const bf16* Xlo = nullptr;
         if (lowrank) {
-            // few rows: the FMA kernel (one launch) beats a K-split tensor-core GEMM plus its reduction
-            cudaError_t e0;
-            if (M <= kFmaDownprojRows && r % 16 == 0) { e0 = stream_downproj_bf16(h, A, M, d, r, c->s.zb, st); n = 1; }
-            else e0 = tensor_downproj(h, A, M, d, r, c->s, c->sm_count, &n, st);
+            // While the call is HBM-bound the tensor cores have time to spare: keep the bf16 rounding
+            // remainder of z and feed it through a second MMA, so z is effectively fp32-exact.
+            const bool low_part = M <= kSplitCodeRows;
+            cudaError_t e0 = tensor_downproj(h, A, M, d, r, low_part, c->s, c->sm_count, &n, st);
             c->launches += n;
             n = 0;
             if (e0 != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
             X = c->s.zb;
+            if (low_part) Xlo = c->s.zb_lo;
         }
-        cudaError_t e = tensor_head(X, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, lowrank, &n, st);
+        cudaError_t e = tensor_head(X, Xlo, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, lowrank, &n, st);
         c->launches += n;
         if (e != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         return SLIMSPEC_OK;

@@ -15,6 +15,7 @@ typedef __nv_bfloat16 bf16;
 struct Scratch {
     float* z;            // fp32 code (or widened h); generic path [M][K], streaming path transposed [K][mt]
     bf16* zb;            // bf16 code [M][r] for the tensor-core path
+    bf16* zb_lo;         // its rounding remainder (z - zb), bf16: used while the call is HBM-bound
     float* zpart;        // K-split partial tiles of the tensor-core down-projection
     size_t zpart_elems;
     uint32_t* smax;      // tensor path: per-row maxima of the sample tiles [64][M padded to 128]
@@ -47,8 +48,6 @@ StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count);
 // z^T = (h A)^T for M <= 8 rows, rows M..mt-1 zero-filled; r must be a multiple of 16.
 cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
                             cudaStream_t st);
-// z (bf16 [M][r]) = h A with FP32 FMAs, any M (A is re-read once per eight rows); r a multiple of 16.
-cudaError_t stream_downproj_bf16(const bf16* h, const bf16* A, int M, int d, int r, bf16* zb, cudaStream_t st);
 // z^T = widened h^T (full-rank head: no down-projection).
 cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st);
 // logits = z B streamed once; mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
@@ -59,13 +58,14 @@ cudaError_t stream_head(const float* z, const bf16* B, int M, int mt, int K, int
 // ---- tensor-core path (larger M) ------------------------------------------------------
 // Shapes the tcgen05 kernels take: K a multiple of 64, N a multiple of 8 and >= 64, k <= 32 in top-k mode.
 bool tensor_ok(int M, int K, int N, int k, int mode);
-// z (bf16 [M][r], in s.zb) = h A.
-cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, const Scratch& s, int sm_count,
-                            int* launches, cudaStream_t st);
+// z (bf16 [M][r], in s.zb) = h A; with_low_part also writes s.zb_lo = bf16(z - zb).
+cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, bool with_low_part, const Scratch& s,
+                            int sm_count, int* launches, cudaStream_t st);
 // X W with X bf16 [M][K], W bf16 [K][N]; mode 0: fused log-softmax / top-k, mode 1: raw fp32 logits.
 // after_kernel: X is written by the kernel launched just before on `st` (the first kernel here is
 // then launched as its programmatic dependent).
-cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
+// Xlo, if not null, is added to X inside the contraction (two MMAs per step).
+cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
                         float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
                         cudaStream_t st);
 

@@ -131,16 +131,11 @@ __device__ __forceinline__ void sort8(uint32_t (&k)[9], int (&i)[9])
 // z^T = (h A)^T for M <= MT rows.  A CTA owns 16 columns of A (two 16-byte units) over all d
 // rows, so no partial sums cross CTAs; a thread owns one unit and every (NT/2)-th row, with
 // RB row loads in flight at a time.  Rows M..MT-1 of z^T are written as zeros.
-// With zb set, blockIdx.y picks a group of MT rows and the result goes to zb[M][r] as bf16 (the
-// operand layout of the tensor-core path) instead of z^T.
 template <int MT, int NT, int RB>
 __global__ void __launch_bounds__(NT) k_stream_downproj(const bf16* __restrict__ h, const bf16* __restrict__ A, int M,
-                                                         int d, int r, float* __restrict__ zT, bf16* __restrict__ zb)
+                                                         int d, int r, float* __restrict__ zT)
 {
     pdl_launch_dependents();
-    const int m0 = blockIdx.y * MT;
-    h += (size_t)m0 * d;
-    M -= m0;
     __shared__ float red[NT / 32][MT][16];
     const int t = threadIdx.x, u = t & 1, rl = t >> 1, lane = t & 31, warp = t >> 5;
     const int c0 = blockIdx.x * 16 + u * 8;
@@ -200,8 +195,7 @@ __global__ void __launch_bounds__(NT) k_stream_downproj(const bf16* __restrict__
         float v = 0.f;
 #pragma unroll
         for (int w = 0; w < NT / 32; ++w) v += red[w][m][c];
-        if (zb == nullptr) zT[(size_t)(blockIdx.x * 16 + c) * MT + m] = v;
-        else if (m < M) zb[(size_t)(m0 + m) * r + blockIdx.x * 16 + c] = __float2bfloat16_rn(v);
+        zT[(size_t)(blockIdx.x * 16 + c) * MT + m] = v;
     }
 }
 
@@ -627,20 +621,11 @@ cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, 
 {
     const int grid = r / 16;
     switch (mt) {
-    case 1: k_stream_downproj<1, 1024, 8><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z, nullptr); break;
-    case 2: k_stream_downproj<2, 1024, 4><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z, nullptr); break;
-    case 4: k_stream_downproj<4, 512, 8><<<grid, 512, 0, st>>>(h, A, M, d, r, s.z, nullptr); break;
-    default: k_stream_downproj<8, 256, 8><<<grid, 256, 0, st>>>(h, A, M, d, r, s.z, nullptr); break;
+    case 1: k_stream_downproj<1, 1024, 8><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z); break;
+    case 2: k_stream_downproj<2, 1024, 4><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z); break;
+    case 4: k_stream_downproj<4, 512, 8><<<grid, 512, 0, st>>>(h, A, M, d, r, s.z); break;
+    default: k_stream_downproj<8, 256, 8><<<grid, 256, 0, st>>>(h, A, M, d, r, s.z); break;
     }
-    return cudaGetLastError();
-}
-
-// z (bf16 [M][r]) = h A on the FP32 pipes, eight rows per CTA row group: for the few-row end of
-// the tensor-core path, where a tensor-core GEMM over d would leave most SMs idle.
-cudaError_t stream_downproj_bf16(const bf16* h, const bf16* A, int M, int d, int r, bf16* zb, cudaStream_t st)
-{
-    dim3 grid(r / 16, (M + 7) / 8);
-    k_stream_downproj<8, 256, 8><<<grid, 256, 0, st>>>(h, A, M, d, r, nullptr, zb);
     return cudaGetLastError();
 }
 

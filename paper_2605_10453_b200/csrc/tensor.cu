@@ -28,6 +28,7 @@ static constexpr float kLog2e = 1.4426950408889634f;
 struct alignas(64) TcParams {
     CUtensorMap mapX;       // X[M][K]: box 64 (K) x 128 rows, 128-byte swizzle
     CUtensorMap mapW;       // W[K][N]: box 64 (N) x 64 (K), 128-byte swizzle
+    CUtensorMap mapX2;      // split mode: the low part of X, same shape and box as mapX
     int M, K, N;
     int nrb, nct, nks;      // row blocks, column tiles, K splits
     int chunks_per_split;   // K chunks of 64 per split
@@ -38,7 +39,11 @@ struct alignas(64) TcParams {
     const uint32_t* thr0;   // mode 0: per-row lower bound (key - 1) of the k-th largest logit, or null
     int k;
     int rec_words;
-    int ns;                 // ring stages
+    int ns;                 // stages of the W ring
+    int nsx;                // stages of the X ring (unused when X is resident)
+    int xbox_bytes;         // bytes of one X box: (rows of the box, 8..128) x 128; rows past the box are garbage in,
+                            // garbage out, and belong to no live row
+    int split;              // 1: X = X_hi + X_lo (two bf16 matrices): two MMAs per step into one accumulator
     int xres;               // 1: the row block's whole X (K <= 512) is loaded once and stays in shared memory
     float* out;
     float* part;            // records [M][2 * gct][rec_words]: two column halves per CTA
@@ -79,24 +84,25 @@ template <int NV>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant__ TcParams p)
 {
     constexpr int NSMAX = 8;                                // most ring stages
-    constexpr int X_BYTES = kTcRows * kTcKChunk * 2;        // 16 KB
     constexpr int WBOX_BYTES = kTcKChunk * 64 * 2;          // 8 KB: 64 k x 64 columns
     constexpr int W_BYTES = WBOX_BYTES * (NV / 64);
     const int NS = p.ns;
-    const bool xres = p.xres != 0;
-    // a stage holds a W chunk, and an X chunk in front of it unless X is resident
-    const int STAGE = xres ? W_BYTES : X_BYTES + W_BYTES;
-    const int W_OFF = xres ? 0 : X_BYTES;
+    const bool xres = p.xres != 0, split = p.split != 0;
+    const int XH = p.xbox_bytes;                            // one X box (high or low part) of a K chunk
+    const int XB = split ? 2 * XH : XH;                     // X bytes per K chunk: high part, then low part
+    // Two rings: W chunks (the HBM stream: as many stages as shared memory allows) and, unless X
+    // is resident, X chunks (L2 hits: a few stages do).
+    const int NSX = p.nsx;
     // instruction descriptor: D fp32, A and B bf16, A K-major, B MN-major, N = NV, M = 128
     constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                ((uint32_t)(NV >> 3) << 17) | ((uint32_t)(kTcRows >> 4) << 24);
 
     extern __shared__ unsigned char smem_raw[];
-    __shared__ uint64_t full[NSMAX], empty[NSMAX], acc_full[2], acc_empty[2], x_full;
+    __shared__ uint64_t full[NSMAX], empty[NSMAX], xfull[4], xempty[4], acc_full[2], acc_empty[2], x_full;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     unsigned char* xarea = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    unsigned char* stages = xarea + (xres ? (size_t)p.chunks_per_split * X_BYTES : 0);
+    unsigned char* stages = xarea + (xres ? (size_t)p.chunks_per_split * XB : (size_t)NSX * XB);   // W ring
     volatile int* abort_flag = &abort_s;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -110,12 +116,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < 4; ++s) { mbar_init(&xfull[s], 1); mbar_init(&xempty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 256); }
         mbar_init(&x_full, 1);
         abort_s = 0;
         mbar_fence_init();
         prefetch_tensor_map(&p.mapX);
         prefetch_tensor_map(&p.mapW);
+        if (p.split) prefetch_tensor_map(&p.mapX2);
     }
     if (warp == 1) tmem_alloc(&tmem_base_s, 2 * NV);
     tc_fence_before_sync();
@@ -130,32 +138,43 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
     if (warp == 0) {
         // ================= producer: one thread issues the TMA loads =================
         if (lane == 0) {
-            int it = 0;
+            // ring positions are kept as (slot, phase) pairs: no division on this thread's path
+            int s = 0, ph = 0, sx = 0, phx = 0;
+            bool first = true, firstx = true;       // first lap: the slots start out empty
             bool alive = true;
             if (xres && ntiles > 0) {
-                mbar_arrive_expect_tx(&x_full, (uint32_t)cps * X_BYTES);
-                for (int c = 0; c < cps; ++c)
-                    tma_load_2d(xarea + (size_t)c * X_BYTES, &p.mapX, c * kTcKChunk, rb * kTcRows, &x_full);
+                mbar_arrive_expect_tx(&x_full, (uint32_t)cps * XB);
+                for (int c = 0; c < cps; ++c) {
+                    tma_load_2d(xarea + (size_t)c * XB, &p.mapX, c * kTcKChunk, rb * kTcRows, &x_full);
+                    if (split) tma_load_2d(xarea + (size_t)c * XB + XH, &p.mapX2, c * kTcKChunk, rb * kTcRows, &x_full);
+                }
             }
             for (int t = 0; t < ntiles && alive; ++t) {
                 const int ct = cg + t * p.gct;
-                for (int c = 0; c < cps; ++c, ++it) {
-                    const int s = it % NS, use = it / NS;
-                    if (use > 0 && !mbar_wait(&empty[s], (use - 1) & 1, abort_flag, p.err, ERR_WAIT_EMPTY)) { alive = false; break; }
-                    unsigned char* st = stages + (size_t)s * STAGE;
-                    mbar_arrive_expect_tx(&full[s], (uint32_t)STAGE);
+                for (int c = 0; c < cps; ++c) {
                     const int kx = (ks * cps + c) * kTcKChunk;
-                    if (!xres) tma_load_2d(st, &p.mapX, kx, rb * kTcRows, &full[s]);
+                    if (!xres) {
+                        if (!firstx && !mbar_wait(&xempty[sx], phx ^ 1, abort_flag, p.err, ERR_WAIT_EMPTY)) { alive = false; break; }
+                        unsigned char* xs = xarea + (size_t)sx * XB;
+                        mbar_arrive_expect_tx(&xfull[sx], (uint32_t)XB);
+                        tma_load_2d(xs, &p.mapX, kx, rb * kTcRows, &xfull[sx]);
+                        if (split) tma_load_2d(xs + XH, &p.mapX2, kx, rb * kTcRows, &xfull[sx]);
+                        if (++sx == NSX) { sx = 0; phx ^= 1; firstx = false; }
+                    }
+                    if (!first && !mbar_wait(&empty[s], ph ^ 1, abort_flag, p.err, ERR_WAIT_EMPTY)) { alive = false; break; }
+                    unsigned char* st = stages + (size_t)s * W_BYTES;
+                    mbar_arrive_expect_tx(&full[s], (uint32_t)W_BYTES);
 #pragma unroll
                     for (int i = 0; i < NV / 64; ++i)
-                        tma_load_2d(st + W_OFF + i * WBOX_BYTES, &p.mapW, ct * NV + i * 64, kx, &full[s]);
+                        tma_load_2d(st + i * WBOX_BYTES, &p.mapW, ct * NV + i * 64, kx, &full[s]);
+                    if (++s == NS) { s = 0; ph ^= 1; first = false; }
                 }
             }
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            int it = 0;
+            int s = 0, ph = 0, sx = 0, phx = 0;
             bool alive = true;
             if (xres && ntiles > 0 && !mbar_wait(&x_full, 0, abort_flag, p.err, ERR_WAIT_FULL)) alive = false;
             for (int t = 0; t < ntiles && alive; ++t) {
@@ -163,21 +182,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 if (t >= 2 && !mbar_wait(&acc_empty[buf], ((t >> 1) - 1) & 1, abort_flag, p.err, ERR_WAIT_FREE)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NV);
-                for (int c = 0; c < cps; ++c, ++it) {
-                    const int s = it % NS, use = it / NS;
-                    if (!mbar_wait(&full[s], use & 1, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
+                for (int c = 0; c < cps; ++c) {
+                    if (!xres && !mbar_wait(&xfull[sx], phx, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
+                    if (!mbar_wait(&full[s], ph, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
                     tc_fence_after_sync();
-                    const uint32_t sa = smem_u32(stages + (size_t)s * STAGE);
-                    const uint32_t xa = xres ? smem_u32(xarea + (size_t)c * X_BYTES) : sa;
+                    const uint32_t sa = smem_u32(stages + (size_t)s * W_BYTES);
+                    const uint32_t xa = smem_u32(xarea + (size_t)(xres ? c : sx) * XB);
                     const uint64_t a_desc = tc_smem_desc_sw128(xa, 16, 1024);
-                    const uint64_t b_desc = tc_smem_desc_sw128(sa + W_OFF, WBOX_BYTES, 1024);
+                    const uint64_t a2_desc = tc_smem_desc_sw128(xa + XH, 16, 1024);
+                    const uint64_t b_desc = tc_smem_desc_sw128(sa, WBOX_BYTES, 1024);
 #pragma unroll
                     for (int j = 0; j < kTcKChunk / 16; ++j) {
                         // 16 of K per instruction: 32 bytes along a K-major row, two 8-row groups of the N-major tile
                         tc_mma_bf16(d_tmem, a_desc + (uint64_t)(j * 2), b_desc + (uint64_t)(j * 128), IDESC,
                                     (c > 0 || j > 0) ? 1u : 0u);
+                        if (split) tc_mma_bf16(d_tmem, a2_desc + (uint64_t)(j * 2), b_desc + (uint64_t)(j * 128), IDESC, 1u);
                     }
                     tc_commit(&empty[s]);
+                    if (++s == NS) { s = 0; ph ^= 1; }
+                    if (!xres) {
+                        tc_commit(&xempty[sx]);
+                        if (++sx == NSX) { sx = 0; phx ^= 1; }
+                    }
                 }
                 if (alive) tc_commit(&acc_full[buf]);
             }
@@ -313,8 +339,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
 }
 
 // ------------------------------------------------------------------------------------------
-// z = sum of the K-split partial tiles, rounded once to bf16.
-__global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad, int M, int r, bf16* __restrict__ z)
+// z = sum of the K-split partial tiles, rounded once to bf16; with zlo set, the rounding error is
+// kept as a second bf16 matrix (z = z + zlo to about 2^-17 relative).
+__global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad, int M, int r, bf16* __restrict__ z,
+                              bf16* __restrict__ zlo)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -329,7 +357,9 @@ __global__ void k_tc_reduce_z(const float* __restrict__ part, int nks, int mpad,
 #pragma unroll
         for (int q = 0; q < 8; ++q) acc += t[q];
     }
-    z[e] = __float2bfloat16_rn(acc);
+    const bf16 hi = __float2bfloat16_rn(acc);
+    z[e] = hi;
+    if (zlo != nullptr) zlo[e] = __float2bfloat16_rn(acc - __bfloat162float(hi));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -470,7 +500,7 @@ bool tensor_ok(int M, int K, int N, int k, int mode)
     return true;
 }
 
-static constexpr size_t kTcSmemMax = 227 * 1024;
+static constexpr size_t kTcSmemMax = 227 * 1024 - 512;   // dynamic shared memory per CTA (a little static on top)
 
 // Launch with (or without) the programmatic-dependent-launch attribute: the kernel may start while
 // the one before it in the stream is still running and meets it at griddepcontrol.wait.
@@ -495,11 +525,12 @@ static cudaError_t launch_chain(void (*kern)(KArgs...), int grid, int block, siz
 template <int NV>
 static cudaError_t launch_gemm(TcParams p, int grid, bool pdl, cudaStream_t st)
 {
-    const size_t x_bytes = (size_t)kTcRows * kTcKChunk * 2, w_bytes = (size_t)kTcKChunk * NV * 2;
+    const size_t x_bytes = (size_t)p.xbox_bytes * (p.split ? 2 : 1), w_bytes = (size_t)kTcKChunk * NV * 2;
     const size_t x_all = (size_t)p.chunks_per_split * x_bytes;
     p.xres = (p.nks == 1 && x_all + 3 * w_bytes + 1024 <= kTcSmemMax) ? 1 : 0;
-    const size_t stage = p.xres ? w_bytes : x_bytes + w_bytes;
-    const size_t fixed = 1024 + (p.xres ? x_all : 0);
+    p.nsx = 4;
+    const size_t fixed = 1024 + (p.xres ? x_all : (size_t)p.nsx * x_bytes);
+    const size_t stage = w_bytes;
     int ns = (int)((kTcSmemMax - fixed) / stage);
     if (ns > 8) ns = 8;
     if (ns < 2) return cudaErrorInvalidValue;
@@ -513,14 +544,21 @@ static cudaError_t launch_gemm(TcParams p, int grid, bool pdl, cudaStream_t st)
 
 // out = X W through the tensor cores.  mode 0: top-k records then merge into ids / logprobs;
 // mode 1: fp32 logits.  X is bf16 [M][K], W bf16 [K][N].
-cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
+cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
                         float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
                         cudaStream_t st)
 {
     TcParams p;
     memset(&p, 0, sizeof(p));
-    if (!make_map(&p.mapX, X, M, K, kTcKChunk, kTcRows) || !make_map(&p.mapW, W, K, N, 64, kTcKChunk))
+    // a single row block loads only as many rows of X as there are (in whole groups of eight)
+    const int xrows = M >= kTcRows ? kTcRows : (M + 7) / 8 * 8;
+    if (!make_map(&p.mapX, X, M, K, kTcKChunk, xrows) || !make_map(&p.mapW, W, K, N, 64, kTcKChunk))
         return cudaErrorInvalidValue;
+    if (Xlo != nullptr) {
+        if (!make_map(&p.mapX2, Xlo, M, K, kTcKChunk, xrows)) return cudaErrorInvalidValue;
+        p.split = 1;
+    }
+    p.xbox_bytes = xrows * kTcKChunk * 2;
     p.M = M; p.K = K; p.N = N;
     p.nrb = (M + kTcRows - 1) / kTcRows;
     const int nv = (p.nrb == 1) ? 128 : 256;
@@ -574,13 +612,15 @@ cudaError_t tensor_head(const bf16* X, const bf16* W, int M, int K, int N, int k
 }
 
 // z (bf16, [M][r]) = h A through the tensor cores: K-split partial tiles, then one reduction.
-cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, const Scratch& s, int sm_count,
-                            int* launches, cudaStream_t st)
+cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, bool with_low_part, const Scratch& s,
+                            int sm_count, int* launches, cudaStream_t st)
 {
     TcParams p;
     memset(&p, 0, sizeof(p));
-    if (!make_map(&p.mapX, h, M, d, kTcKChunk, kTcRows) || !make_map(&p.mapW, A, d, r, 64, kTcKChunk))
+    const int xrows = M >= kTcRows ? kTcRows : (M + 7) / 8 * 8;
+    if (!make_map(&p.mapX, h, M, d, kTcKChunk, xrows) || !make_map(&p.mapW, A, d, r, 64, kTcKChunk))
         return cudaErrorInvalidValue;
+    p.xbox_bytes = xrows * kTcKChunk * 2;
     p.M = M; p.K = d; p.N = r;
     p.nrb = (M + kTcRows - 1) / kTcRows;
     p.nct = (r + 127) / 128;
@@ -602,7 +642,7 @@ cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, c
     if (e != cudaSuccess) return e;
     const int n = M * r;
     e = launch_chain(k_tc_reduce_z, (n + 255) / 256, 256, 0, true, st, (const float*)s.zpart, nks, p.nrb * kTcRows, M, r,
-                     s.zb);
+                     s.zb, with_low_part ? s.zb_lo : (bf16*)nullptr);
     *launches += 2;
     return e;
 }

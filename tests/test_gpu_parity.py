@@ -189,12 +189,16 @@ def test_throughput_batch_sampled_rows(ctx):
     c = synth.CONFIGS["c3"]
     x = synth.make_inputs(M, c.d, c.r, c.V, seed=c.seed)
     g = dev(x)
-    # (same kernels for the single row, so that only the batch around it changes)
-    ctx.force_path(binding.PATH_TENSOR)
-    for m in (5, 200, 300, 509):
-        i1, l1 = ctx.slimspec_head_topk(g["h"][m:m + 1].contiguous(), g["A"], g["B"], c.k)
-        assert np.array_equal(i1.cpu().numpy()[0], ids[m])
-        assert np.max(np.abs(l1.cpu().numpy()[0] - lp[m])) < 2e-4
+    # (a sub-batch that takes the same kernels in the same precision mode -- more than 256 rows --
+    # but puts every row at another position of another 128-row tile)
+    m0 = 200
+    i1, l1 = ctx.slimspec_head_topk(g["h"][m0:].contiguous(), g["A"], g["B"], c.k)
+    torch.cuda.synchronize()
+    assert ctx.last_path() == binding.PATH_TENSOR
+    i1, l1 = i1.cpu().numpy(), l1.cpu().numpy()
+    for m in (200, 300, 383, 384, 509, 511):
+        assert np.array_equal(i1[m - m0], ids[m])
+        assert np.max(np.abs(l1[m - m0] - lp[m])) < 2e-4
 
 
 @pytest.mark.parametrize("r,M", [(1024, 64), (2048, 4)])
