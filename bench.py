@@ -180,6 +180,21 @@ def time_calls(torch, fn, n):
     return e0.elapsed_time(e1)
 
 
+def max_over_ranks(dist, ms, device):
+    """The slowest rank's time: what a job of independent replicas takes.  dist None = one process."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_us_per_call(ms_max, steps, world):
+    """Whole-job microseconds per call: `world` replicas finish steps * world calls in ms_max."""
+    return ms_max * 1e3 / (steps * world)
+
+
 def copies_needed(nbytes):
     return max(2, -(-4 * L2_BYTES // nbytes))
 
@@ -227,13 +242,6 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
-
     K, W = args.steps, max(args.warmup, 3)
     sampler = ClockSampler(local)
     for i in range(W):
@@ -245,7 +253,7 @@ def run_ours(args):
     ms = time_calls(torch, step, K)
     launches = ctx.launch_count() - n0
     barrier()
-    ms = max_over_ranks(ms)
+    ms = max_over_ranks(dist, ms, dev)
     # ---- the dominant kernel alone, events recorded by the library around it, same K steps
     ctx.kernel_timing(True)
     for i in range(K):
@@ -256,13 +264,13 @@ def run_ours(args):
     for i in range(3):
         step_host(i)
     barrier()
-    e2e_ms = max_over_ranks(time_calls(torch, step_host, K))
+    e2e_ms = max_over_ranks(dist, time_calls(torch, step_host, K), dev)
     clocks = sampler.stop()
     if ctx.last_error() != binding.OK:
         raise SystemExit("device-side wait timed out during the benchmark")
 
-    us_call = ms * 1e3 / (K * world)
-    e2e_us = e2e_ms * 1e3 / (K * world)
+    us_call = job_us_per_call(ms, K, world)
+    e2e_us = job_us_per_call(e2e_ms, K, world)
     kern_us = kms * 1e3 / max(kn, 1)
     kern_bytes = 2 * r * V + 4 * r * M            # the streamed matrix and the fp32 code
     achieved = kern_bytes / (kern_us * 1e-6) / 1e9
