@@ -14,14 +14,27 @@ NVCC_FLAGS = [
 ]
 
 
-def _newest_source_mtime() -> float:
-    paths = [os.path.join(_CSRC, f) for f in os.listdir(_CSRC)]
+STAMP_PATH = os.path.join(_PKG, "libslimspec.srchash")
+
+
+def _source_hash() -> str:
+    """SHA-256 over the sources the library is built from (file times do not survive a copy)."""
+    import hashlib
+    h = hashlib.sha256()
+    paths = sorted(os.path.join(_CSRC, f) for f in os.listdir(_CSRC))
     paths.append(os.path.join(os.path.dirname(_PKG), "include", "slimspec.h"))
-    return max(os.path.getmtime(p) for p in paths)
+    for p in paths:
+        h.update(os.path.basename(p).encode())
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def is_stale() -> bool:
-    return (not os.path.exists(LIB_PATH)) or os.path.getmtime(LIB_PATH) < _newest_source_mtime()
+    if not (os.path.exists(LIB_PATH) and os.path.exists(STAMP_PATH)):
+        return True
+    with open(STAMP_PATH) as f:
+        return f.read().strip() != _source_hash()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -32,8 +45,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB_PATH + ".tmp%d" % os.getpid()
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp]
     cmd += [os.path.join(_CSRC, s) for s in SOURCES]
+    digest = _source_hash()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)
+    with open(STAMP_PATH + ".tmp%d" % os.getpid(), "w") as f:
+        f.write(digest + "\n")
+    os.replace(STAMP_PATH + ".tmp%d" % os.getpid(), STAMP_PATH)
     return LIB_PATH
 
 
