@@ -22,6 +22,10 @@ static constexpr int kTcKChunk = 64;         // K per stage: 64 bf16 = one 128-b
 static constexpr int kTcThreads = 320;       // TMA warp, MMA warp, eight epilogue warps
 static constexpr int kTcMaxK = 32;           // largest k
 static constexpr int kTcList = 48;           // candidates a row parks before the list is compacted
+static constexpr int kTcListPitch = 49;      // words between two rows' lists in shared memory: odd, so lanes hit distinct banks
+static constexpr int kTcEpiThreads = 256;    // epilogue threads per CTA
+// shared memory the final sort of the lists needs (values and ids of every epilogue thread)
+static constexpr size_t kTcSortBytes = (size_t)2 * kTcEpiThreads * kTcListPitch * 4;
 static constexpr int kTcNoId = 0x7fffffff;
 static constexpr float kLog2e = 1.4426950408889634f;
 
@@ -173,8 +177,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         }
     } else if (warp == 1) {
         // ================= MMA issuer =================
+        // One thread feeds the tensor pipe, so its instruction count per K chunk is what bounds the
+        // main loop once the data is there: descriptors are kept as a running low word (start
+        // address and leading offset; the high word is the same for every operand) and ring
+        // positions as (slot, phase) pairs.
         if (lane == 0) {
+            constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);     // SBO 1024, version 1, 128-byte swizzle
+            const uint32_t a_base = ((smem_u32(xarea) >> 4) & 0x3fffu) | (1u << 16);                       // LBO 16
+            const uint32_t b_base = ((smem_u32(stages) >> 4) & 0x3fffu) | ((uint32_t)(WBOX_BYTES >> 4) << 16);
+            const uint32_t a_step = (uint32_t)XB >> 4, a_lowpart = (uint32_t)XH >> 4;
+            constexpr uint32_t B_STEP = (uint32_t)W_BYTES >> 4;
+            const int nsa = xres ? cps : NSX;           // X slots: the resident chunks, or the ring
             int s = 0, ph = 0, sx = 0, phx = 0;
+            uint32_t a_lo = a_base, b_lo = b_base;
             bool alive = true;
             if (xres && ntiles > 0 && !mbar_wait(&x_full, 0, abort_flag, p.err, ERR_WAIT_FULL)) alive = false;
             for (int t = 0; t < ntiles && alive; ++t) {
@@ -183,27 +198,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * NV);
                 for (int c = 0; c < cps; ++c) {
-                    if (!xres && !mbar_wait(&xfull[sx], phx, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
-                    if (!mbar_wait(&full[s], ph, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
-                    tc_fence_after_sync();
-                    const uint32_t sa = smem_u32(stages + (size_t)s * W_BYTES);
-                    const uint32_t xa = smem_u32(xarea + (size_t)(xres ? c : sx) * XB);
-                    const uint64_t a_desc = tc_smem_desc_sw128(xa, 16, 1024);
-                    const uint64_t a2_desc = tc_smem_desc_sw128(xa + XH, 16, 1024);
-                    const uint64_t b_desc = tc_smem_desc_sw128(sa, WBOX_BYTES, 1024);
+                    if (!xres && !mbar_try_wait(&xfull[sx], phx) && !mbar_wait(&xfull[sx], phx, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
+                    if (!mbar_try_wait(&full[s], ph) && !mbar_wait(&full[s], ph, abort_flag, p.err, ERR_WAIT_FULL)) { alive = false; break; }
+                    // 16 of K per instruction: 32 bytes along a K-major row of X, two 8-row groups of the N-major W tile
+                    tc_mma_bf16_words(d_tmem, a_lo, b_lo, DESC_HI, IDESC, c > 0 ? 1u : 0u);
+                    if (split) tc_mma_bf16_words(d_tmem, a_lo + a_lowpart, b_lo, DESC_HI, IDESC, 1u);
 #pragma unroll
-                    for (int j = 0; j < kTcKChunk / 16; ++j) {
-                        // 16 of K per instruction: 32 bytes along a K-major row, two 8-row groups of the N-major tile
-                        tc_mma_bf16(d_tmem, a_desc + (uint64_t)(j * 2), b_desc + (uint64_t)(j * 128), IDESC,
-                                    (c > 0 || j > 0) ? 1u : 0u);
-                        if (split) tc_mma_bf16(d_tmem, a2_desc + (uint64_t)(j * 2), b_desc + (uint64_t)(j * 128), IDESC, 1u);
+                    for (int j = 1; j < kTcKChunk / 16; ++j) {
+                        tc_mma_bf16_words(d_tmem, a_lo + (uint32_t)(j * 2), b_lo + (uint32_t)(j * 128), DESC_HI, IDESC, 1u);
+                        if (split) tc_mma_bf16_words(d_tmem, a_lo + a_lowpart + (uint32_t)(j * 2), b_lo + (uint32_t)(j * 128), DESC_HI, IDESC, 1u);
                     }
                     tc_commit(&empty[s]);
-                    if (++s == NS) { s = 0; ph ^= 1; }
-                    if (!xres) {
-                        tc_commit(&xempty[sx]);
-                        if (++sx == NSX) { sx = 0; phx ^= 1; }
-                    }
+                    b_lo += B_STEP;
+                    if (++s == NS) { s = 0; ph ^= 1; b_lo = b_base; }
+                    if (!xres) tc_commit(&xempty[sx]);
+                    a_lo += a_step;
+                    if (++sx == nsa) { sx = 0; phx ^= 1; a_lo = a_base; }
                 }
                 if (alive) tc_commit(&acc_full[buf]);
             }
@@ -229,7 +239,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         for (int t = 0; t < ntiles && alive; ++t) {
             const int buf = t & 1;
             const int ct = cg + t * p.gct;
-            if (!mbar_wait(&acc_full[buf], (t >> 1) & 1, abort_flag, p.err, ERR_WAIT_ACC)) { alive = false; break; }
+            if (!mbar_wait_warp(&acc_full[buf], (t >> 1) & 1, abort_flag, p.err, ERR_WAIT_ACC)) { alive = false; break; }
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NV);
             float tile_max = -FLT_MAX;
@@ -321,13 +331,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             mbar_arrive(&acc_empty[buf]);
         }
         if (alive && live && p.mode == 0) {
-            topk_compact(cv, ci, cnt, k, thr);
+            // The lists live in local memory, which this kernel's small L1 hardly caches: a sort
+            // there pays an L2 round trip per step.  Every MMA has completed by now (the last
+            // accumulator was handed over), so the operand rings are dead: sort in that memory.
+            float* sv = reinterpret_cast<float*>(xarea) + (size_t)(tid - 64) * kTcListPitch;
+            int* si = reinterpret_cast<int*>(xarea + (size_t)kTcEpiThreads * kTcListPitch * 4) + (size_t)(tid - 64) * kTcListPitch;
+            for (int j = 0; j < cnt; ++j) {
+                sv[j] = cv[j];
+                si[j] = ci[j];
+            }
+            topk_compact(sv, si, cnt, k, thr);
             float* rec = p.part + ((size_t)m * (2 * p.gct) + 2 * cg + half) * p.rec_words;
             rec[0] = run_max;
             rec[1] = run_sum;
             for (int j = 0; j < k; ++j) {
-                rec[2 + j] = __uint_as_float(j < cnt ? f2key(cv[j] + 0.f) : 0u);      // -0 and +0 rank alike
-                rec[2 + k + j] = __int_as_float(j < cnt ? ci[j] : kTcNoId);
+                rec[2 + j] = __uint_as_float(j < cnt ? f2key(sv[j] + 0.f) : 0u);      // -0 and +0 rank alike
+                rec[2 + k + j] = __int_as_float(j < cnt ? si[j] : kTcNoId);
             }
         }
     }
@@ -535,7 +554,8 @@ static cudaError_t launch_gemm(TcParams p, int grid, bool pdl, cudaStream_t st)
     if (ns > 8) ns = 8;
     if (ns < 2) return cudaErrorInvalidValue;
     p.ns = ns;
-    const size_t smem = fixed + (size_t)ns * stage;
+    size_t smem = fixed + (size_t)ns * stage;
+    if (p.mode == 0 && smem < 1024 + kTcSortBytes) smem = 1024 + kTcSortBytes;      // room for the final sort of the lists
     auto kern = k_tc_gemm<NV>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
