@@ -83,6 +83,121 @@ __device__ __forceinline__ float ex2_fast(float x)
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+// What one epilogue thread carries for its row across the tiles of its CTA.
+struct EpiRow {
+    float run_max, run_sum;     // online softmax: maximum so far, sum of exp(logit - maximum)
+    float thr;                  // candidates must beat this
+    float tile_max;             // mode 3: maximum of the current tile
+    int cnt;                    // candidates parked in the list
+};
+
+// One chunk of 32 consecutive columns of one row, as read from tensor memory.
+__device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&v)[32], int col0, int m, int ks, bool live,
+                                          EpiRow& st, float* cv, int* ci)
+{
+    const int nvalid = min(32, p.N - col0);      // same for every thread
+    if (nvalid <= 0 || !live) return;
+    if (p.mode == 3) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) st.tile_max = fmaxf(st.tile_max, e < nvalid ? __uint_as_float(v[e]) : -FLT_MAX);
+        return;
+    }
+    if (p.mode != 0) {
+        const size_t orow = (p.mode == 2) ? ((size_t)ks * p.nrb * kTcRows + m) : (size_t)m;
+        float* dst = p.out + orow * p.N + col0;
+#pragma unroll
+        for (int e = 0; e < 32; e += 4) {
+            if (e < nvalid)      // N is a multiple of 8, so a group of four is all in or all out
+                *reinterpret_cast<float4*>(dst + e) =
+                    make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
+                                __uint_as_float(v[e + 3]));
+        }
+        return;
+    }
+    // ---- online softmax and candidate filter.  Columns past N (last tile only) count as -FLT_MAX.
+    float x[32];
+#pragma unroll
+    for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]);
+    if (nvalid < 32) {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) x[e] = e < nvalid ? x[e] : -FLT_MAX;
+    }
+    float m8[4];       // maxima of the four groups of eight columns (three-input max: four steps a group)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        float g = max3(x[q * 8], x[q * 8 + 1], x[q * 8 + 2]);
+        g = max3(g, x[q * 8 + 3], x[q * 8 + 4]);
+        g = max3(g, x[q * 8 + 5], x[q * 8 + 6]);
+        m8[q] = fmaxf(g, x[q * 8 + 7]);
+    }
+    const float cmax = fmaxf(max3(m8[0], m8[1], m8[2]), m8[3]);
+    if (cmax > st.run_max) {
+        st.run_sum *= ex2_fast((st.run_max - cmax) * kLog2e);
+        st.run_max = cmax;
+    }
+    // sum of 2^(x log2(e) - max log2(e)): the scaling and the adds go two columns an instruction
+    const float nmb = -st.run_max * kLog2e;
+    const float2 sc = make_float2(kLog2e, kLog2e), of = make_float2(nmb, nmb);
+    float2 sacc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+    for (int e = 0; e < 32; e += 2) {
+        const float2 t = __ffma2_rn(make_float2(x[e], x[e + 1]), sc, of);
+        sacc[(e >> 1) & 1] = __fadd2_rn(sacc[(e >> 1) & 1], make_float2(ex2_fast(t.x), ex2_fast(t.y)));
+    }
+    st.run_sum += (sacc[0].x + sacc[0].y) + (sacc[1].x + sacc[1].y);
+    // top-k: ids arrive in ascending order, so a candidate must beat the threshold strictly.  Some
+    // row of the warp has a candidate in most chunks, but a given row rarely has one: a lane with
+    // one looks only into the groups of eight whose maximum beats its threshold.  (No warp-wide
+    // vote here: lanes of rows past M have returned.)
+    if (cmax > st.thr) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (m8[q] > st.thr) {
+                uint32_t gt = 0u;       // the group's columns above the threshold, built without branches
+#pragma unroll
+                for (int e = 0; e < 8; ++e) gt |= (x[q * 8 + e] > st.thr) ? (1u << e) : 0u;
+                if ((gt & (gt - 1u)) == 0u) {
+                    // one column: it is the group's maximum
+                    if (st.cnt == kTcList) {
+                        int c = st.cnt;      // a copy: the state stays in registers
+                        st.thr = topk_compact(cv, ci, c, p.k, st.thr);
+                        st.cnt = c;
+                    }
+                    if (m8[q] > st.thr) {
+                        cv[st.cnt] = m8[q];
+                        ci[st.cnt] = col0 + q * 8 + __ffs(gt) - 1;
+                        ++st.cnt;
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const float xv = x[q * 8 + e];
+                        if (xv > st.thr) {
+                            if (st.cnt == kTcList) {
+                                int c = st.cnt;
+                                st.thr = topk_compact(cv, ci, c, p.k, st.thr);
+                                st.cnt = c;
+                            }
+                            if (xv > st.thr) {
+                                cv[st.cnt] = xv;
+                                ci[st.cnt] = col0 + q * 8 + e;
+                                ++st.cnt;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 template <int NV>
 __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant__ TcParams p)
@@ -226,110 +341,39 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         const int m = rb * kTcRows + row;
         const bool live = m < p.M;
         const int k = p.k;
-        float run_max = -FLT_MAX, run_sum = 0.f;
+        EpiRow st;
+        st.run_max = -FLT_MAX;
+        st.run_sum = 0.f;
+        st.cnt = 0;
         float cv[kTcList];
         int ci[kTcList];
-        int cnt = 0;
         // Candidates must beat thr: the k-th best value once the list is full, before that a bound
         // known to lie below the row's k-th largest logit (from a sample of the vocabulary).
         const uint32_t thr0_key = (p.mode == 0 && p.thr0 != nullptr && live) ? __ldg(p.thr0 + m) : 0u;
-        const float thr0 = thr0_key != 0u ? key2f(thr0_key) : -FLT_MAX;      // key 0: no bound
-        float thr = thr0;
+        st.thr = thr0_key != 0u ? key2f(thr0_key) : -FLT_MAX;      // key 0: no bound
         bool alive = true;
+        constexpr int NCH = NV / 2 / 32;          // chunks of 32 columns per warp and tile: 2 or 4
         for (int t = 0; t < ntiles && alive; ++t) {
             const int buf = t & 1;
             const int ct = cg + t * p.gct;
             if (!mbar_wait_warp(&acc_full[buf], (t >> 1) & 1, abort_flag, p.err, ERR_WAIT_ACC)) { alive = false; break; }
             tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NV);
-            float tile_max = -FLT_MAX;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * NV + half * (NV / 2));
+            const int colbase = ct * NV + half * (NV / 2);
+            st.tile_max = -FLT_MAX;
 #pragma unroll 1
-            for (int c0 = half * (NV / 2); c0 < (half + 1) * (NV / 2); c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32x32(taddr + (uint32_t)c0, v);
+            for (int i = 0; i < NCH; ++i) {
+                uint32_t va[32];
+                tmem_ld_32x32(taddr + (uint32_t)(i * 32), va);
                 tmem_ld_wait();
-                const int col0 = ct * NV + c0;
-                const int nvalid = min(32, p.N - col0);      // same for every thread
-                if (nvalid <= 0 || !live) continue;
-                if (p.mode == 3) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) tile_max = fmaxf(tile_max, e < nvalid ? __uint_as_float(v[e]) : -FLT_MAX);
-                    continue;
-                }
-                if (p.mode != 0) {
-                    const size_t orow = (p.mode == 2) ? ((size_t)ks * p.nrb * kTcRows + m) : (size_t)m;
-                    float* dst = p.out + orow * p.N + col0;
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        if (e < nvalid)      // N is a multiple of 8, so a group of four is all in or all out
-                            *reinterpret_cast<float4*>(dst + e) =
-                                make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]), __uint_as_float(v[e + 2]),
-                                            __uint_as_float(v[e + 3]));
-                    }
-                    continue;
-                }
-                // ---- online softmax and candidate filter; four independent chains keep the one
-                // warp of this scheduler busy.  Columns past N (last tile only) count as -FLT_MAX.
-                float x[32];
-#pragma unroll
-                for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(v[e]);
-                if (nvalid < 32) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) x[e] = e < nvalid ? x[e] : -FLT_MAX;
-                }
-                float m8[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    m8[q] = x[q * 8];
-#pragma unroll
-                    for (int e = 1; e < 8; ++e) m8[q] = fmaxf(m8[q], x[q * 8 + e]);
-                }
-                const float cmax = fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3]));
-                if (cmax > run_max) {
-                    run_sum *= ex2_fast((run_max - cmax) * kLog2e);
-                    run_max = cmax;
-                }
-                const float mb = run_max * kLog2e;
-                float sacc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int e = 0; e < 32; ++e) sacc[e & 3] += ex2_fast(fmaf(x[e], kLog2e, -mb));
-                run_sum += (sacc[0] + sacc[1]) + (sacc[2] + sacc[3]);
-                // top-k: ids arrive in ascending order, so a candidate must beat the threshold strictly.
-                // Some row of the warp has a candidate in most chunks, but a given row rarely has
-                // one and hardly ever two.  So a lane with a candidate builds the bit mask of its
-                // columns above its threshold with straight-line code; a single set bit is the chunk
-                // maximum and is appended without indexing registers; only two or more take the
-                // branchy scan.
-                if (cmax > thr) {      // no warp-wide vote here: lanes of rows past M have left the loop body
-                    uint32_t gt = 0u;
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) gt |= (x[e] > thr) ? (1u << e) : 0u;
-                    if (gt != 0u) {
-                        if ((gt & (gt - 1u)) == 0u) {
-                            if (cnt == kTcList) thr = topk_compact(cv, ci, cnt, k, thr);
-                            cv[cnt] = cmax;
-                            ci[cnt] = col0 + __ffs(gt) - 1;
-                            ++cnt;
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) {
-                                if (x[e] > thr) {
-                                    if (cnt == kTcList) thr = topk_compact(cv, ci, cnt, k, thr);
-                                    if (x[e] > thr) {
-                                        cv[cnt] = x[e];
-                                        ci[cnt] = col0 + e;
-                                        ++cnt;
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
+                epi_chunk(p, va, colbase + i * 32, m, ks, live, st, cv, ci);
             }
-            if (p.mode == 3 && live) p.smax[((size_t)ct * 2 + half) * p.nrb * kTcRows + m] = f2key(tile_max);
+            if (p.mode == 3 && live) p.smax[((size_t)ct * 2 + half) * p.nrb * kTcRows + m] = f2key(st.tile_max);
             tc_fence_before_sync();
             mbar_arrive(&acc_empty[buf]);
         }
+        const float run_max = st.run_max, run_sum = st.run_sum, thr = st.thr;
+        int cnt = st.cnt;
         if (alive && live && p.mode == 0) {
             // The lists live in local memory, which this kernel's small L1 hardly caches: a sort
             // there pays an L2 round trip per step.  Every MMA has completed by now (the last
