@@ -140,6 +140,13 @@ __global__ void __launch_bounds__(NT) k_stream_downproj(const bf16* __restrict__
     const int t = threadIdx.x, u = t & 1, rl = t >> 1, lane = t & 31, warp = t >> 5;
     const int c0 = blockIdx.x * 16 + u * 8;
     constexpr int RSTEP = NT / 2;
+    // Launched early (programmatic dependent launch), this kernel may start while the kernel before
+    // it in the stream is still finishing: until that one is complete it only asks the L2 for its
+    // slice of A (a hint; no value is read), then it waits.  h and z^T are touched after the wait.
+    if (u == 0) {
+        for (int i = rl; i < d; i += RSTEP) prefetch_l2(A + (size_t)i * r + c0);
+    }
+    pdl_wait();
 
     float acc[MT][8];
 #pragma unroll
@@ -203,6 +210,7 @@ __global__ void __launch_bounds__(NT) k_stream_downproj(const bf16* __restrict__
 __global__ void k_stream_widen_t(const bf16* __restrict__ h, int M, int MT, int d, float* __restrict__ zT)
 {
     pdl_launch_dependents();
+    pdl_wait();          // launched early: the kernel before it may still read z^T
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= d * MT) return;
     const int i = e / MT, m = e % MT;
@@ -270,7 +278,9 @@ __global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const He
             }
     };
     if (npass > 0) prologue(0);
-    // the weights are on their way; now wait for the kernel that writes the code
+    // the weights are on their way; let the next kernel in the stream come up behind this one,
+    // then wait for the kernel that writes the code
+    pdl_launch_dependents();
     if (p.wait_prev) pdl_wait();
 
     float run_max[MT], run_sum[MT];
@@ -616,24 +626,42 @@ StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count)
     return sp;
 }
 
+// Launch with programmatic stream serialization: the kernel may begin once every CTA of the kernel
+// before it in the stream has signalled launch_dependents or left; it orders itself after that
+// kernel with griddepcontrol.wait.  Across calls this hides the launch gap and lets the first
+// kernel of a call warm up under the tail of the last kernel of the call before.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_early(void (*kern)(KArgs...), int grid, int block, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
                             cudaStream_t st)
 {
     const int grid = r / 16;
     switch (mt) {
-    case 1: k_stream_downproj<1, 1024, 8><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z); break;
-    case 2: k_stream_downproj<2, 1024, 4><<<grid, 1024, 0, st>>>(h, A, M, d, r, s.z); break;
-    case 4: k_stream_downproj<4, 512, 8><<<grid, 512, 0, st>>>(h, A, M, d, r, s.z); break;
-    default: k_stream_downproj<8, 256, 8><<<grid, 256, 0, st>>>(h, A, M, d, r, s.z); break;
+    case 1: return launch_early(k_stream_downproj<1, 1024, 8>, grid, 1024, st, h, A, M, d, r, s.z);
+    case 2: return launch_early(k_stream_downproj<2, 1024, 4>, grid, 1024, st, h, A, M, d, r, s.z);
+    case 4: return launch_early(k_stream_downproj<4, 512, 8>, grid, 512, st, h, A, M, d, r, s.z);
+    default: return launch_early(k_stream_downproj<8, 256, 8>, grid, 256, st, h, A, M, d, r, s.z);
     }
-    return cudaGetLastError();
 }
 
 cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st)
 {
     const int n = d * mt;
-    k_stream_widen_t<<<(n + 255) / 256, 256, 0, st>>>(h, M, mt, d, zT);
-    return cudaGetLastError();
+    return launch_early(k_stream_widen_t, (n + 255) / 256, 256, st, h, M, mt, d, zT);
 }
 
 template <int MT, int U>

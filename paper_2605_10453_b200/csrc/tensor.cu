@@ -457,6 +457,7 @@ static constexpr int kMergeLists = 10;
 __global__ void __launch_bounds__(128) k_tc_merge(const float* __restrict__ part, int M, int P, int RW, int k,
                                                   int32_t* __restrict__ ids, float* __restrict__ logprobs)
 {
+    pdl_launch_dependents();     // the first kernel of the next call may come up behind this one
     pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m = blockIdx.x * (blockDim.x >> 5) + warp;
@@ -612,6 +613,9 @@ cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, in
                         float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
                         cudaStream_t st)
 {
+    // Every kernel here orders itself after its predecessor with griddepcontrol.wait before it touches
+    // global memory, so each one, the first included, is launched early.
+    after_kernel = true;
     TcParams p;
     memset(&p, 0, sizeof(p));
     // a single row block loads only as many rows of X as there are (in whole groups of eight)
@@ -702,7 +706,9 @@ cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, b
     p.err = s.err;
     const size_t need = (size_t)nks * p.nrb * kTcRows * r;
     if (need > s.zpart_elems) return cudaErrorInvalidValue;
-    cudaError_t e = launch_gemm<128>(p, p.nrb * p.nct * nks, false, st);
+    // Launched early even as the first kernel of a call: it touches global memory only after its
+    // griddepcontrol.wait, so it may come up under the tail of whatever kernel precedes it.
+    cudaError_t e = launch_gemm<128>(p, p.nrb * p.nct * nks, true, st);
     if (e != cudaSuccess) return e;
     const int n = M * r;
     e = launch_chain(k_tc_reduce_z, (n + 255) / 256, 256, 0, true, st, (const float*)s.zpart, nks, p.nrb * kTcRows, M, r,
