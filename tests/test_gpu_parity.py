@@ -322,3 +322,35 @@ def test_argument_errors_launch_nothing(ctx):
     assert call(513, 64, 64, 800, 4) == binding.ERR_DIM
     assert call(2, 64, 64, 200008, 4) == binding.ERR_DIM
     assert ctx.launch_count() == n0
+
+
+# ---------------------------------------------------------------- calls in a row, no host synchronisation
+
+@pytest.mark.parametrize("M", [1, 3, 12])
+def test_back_to_back_calls_keep_stream_order(ctx, M):
+    """Kernels of one call are launched early behind the kernels of the call before (and behind
+    whatever else precedes them in the stream).  Ten calls in a row, with no host synchronisation,
+    alternate between two different inputs whose h is written by another kernel on the same stream
+    just before each call; every result must equal that of the same call made alone."""
+    ctx.force_path(binding.PATH_AUTO)
+    d, r, V, k = 1024, 128, 32 * 1024, 10
+    xs = [dev(synth.make_inputs(M, d, r, V, seed=71 + i)) for i in range(2)]
+    alone = []
+    for x in xs:
+        ids, lp = ctx.slimspec_head_topk(x["h"], x["A"], x["B"], k)
+        torch.cuda.synchronize()
+        alone.append((ids.clone(), lp.clone()))
+    n = 10
+    out_ids = [torch.full((M, k), -7, dtype=torch.int32, device=DEV) for _ in range(n)]
+    out_lp = [torch.zeros((M, k), dtype=torch.float32, device=DEV) for _ in range(n)]
+    hbuf = torch.zeros_like(xs[0]["h"])
+    for i in range(n):
+        x = xs[i % 2]
+        hbuf.copy_(x["h"])            # a kernel on the same stream writes the call's input
+        ctx.slimspec_head_topk(hbuf, x["A"], x["B"], k, out_ids=out_ids[i], out_logprobs=out_lp[i])
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK
+    for i in range(n):
+        ids, lp = alone[i % 2]
+        assert torch.equal(out_ids[i], ids), "call %d" % i
+        assert torch.equal(out_lp[i], lp), "call %d" % i
