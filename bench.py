@@ -387,6 +387,40 @@ def extra_points(torch, ctx, synth, binding, dev, peaks):
     return out
 
 
+def run_point(args):
+    """One other point of the metric by itself (the 8B-class shapes at --point M rows, cold rotating
+    weights, --warmup untimed then --steps timed calls): the command the profiler captures are made with."""
+    import torch
+    from paper_2605_10453_b200 import binding, build, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    build.build()
+    peaks, kind = load_peaks()
+    c1 = synth.CONFIGS["c1"]
+    d, r, V, k, M = c1.d, c1.r, c1.V, c1.k, args.point
+    x = synth.make_inputs(8, d, r, V, seed=c1.seed)
+    R = copies_needed(2 * (d * r + r * V))
+    As = [x["A"].to(dev).clone() for _ in range(R)]
+    Bs = [x["B"].to(dev).clone() for _ in range(R)]
+    ctx = binding.Context(max_M=max(M, 8), max_d=d, max_V=V, max_k=k)
+    h = synth.make_h(M, d, c1.seed).to(dev)
+    ids = torch.empty((M, k), dtype=torch.int32, device=dev)
+    lp = torch.empty((M, k), dtype=torch.float32, device=dev)
+    fn = lambda i: ctx.slimspec_head_topk(h, As[i % R], Bs[i % R], k, out_ids=ids, out_logprobs=lp)
+    for i in range(max(args.warmup, 3)):
+        fn(i)
+    us = time_calls(torch, fn, args.steps) * 1e3 / args.steps
+    if ctx.last_error() != binding.OK:
+        raise RuntimeError("device-side wait timed out")
+    t_hbm = head_bytes(M, d, r, V, k) / (peaks["hbm_gbs"] * 1e9)
+    t_mma = head_flops(M, d, r, V) / (peaks["bf16_tflops"] * 1e12)
+    print(json.dumps({"point": "c1 shapes, M=%d" % M, "us_per_call": us, "rows_per_s": M / (us * 1e-6),
+                      "roofline_us": max(t_hbm, t_mma) * 1e6, "roofline_frac": max(t_hbm, t_mma) * 1e6 / us,
+                      "bound": "hbm" if t_hbm >= t_mma else "tensor", "peaks": kind, "steps": args.steps,
+                      "path": {1: "generic", 2: "stream", 3: "tensor"}.get(ctx.last_path(), "?")}))
+    ctx.close()
+
+
 def run_sweep(args):
     """The rank / batch sweep (d=8192, V=128256, r in {d/16, d/8, d/4} and full rank, M in {1..1024}):
     one JSON line per point with us/call and the fraction of the roofline, then a markdown table.
@@ -459,9 +493,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the extra points and the CPU baseline")
     ap.add_argument("--sweep", action="store_true", help="run the rank / batch sweep instead of the benchmark line")
+    ap.add_argument("--point", type=int, default=0, metavar="M",
+                    help="time only the 8B-class shapes at M rows (for profiler captures) instead of the benchmark line")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+    elif args.point > 0:
+        run_point(args)
     elif args.impl == "reference":
         run_reference(args)
     else:
