@@ -16,7 +16,11 @@ struct slimspec_ctx {
     long long launches;
     Scratch s;
     bf16* h_stage;        // device copy of host activations (head_topk_host)
-    int32_t* ids_stage;   // device results of head_topk_host
+    // Results of head_topk_host: pinned host memory mapped into the device, so the kernels write
+    // them straight to the host (80 bytes at M = 1) and no device-to-host copy is enqueued.
+    void* res_host;       // host address of the mapping: ids, then log-probs
+    size_t res_half;      // bytes from the ids to the log-probs
+    int32_t* ids_stage;   // device addresses of the same memory
     float* lp_stage;
     // optional device timing of the kernel that streams the weight matrix
     int timing_on;
@@ -91,8 +95,17 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     ok = ok && cudaMalloc(&c->s.tickets, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.err, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->h_stage, (size_t)max_M * max_d * sizeof(bf16)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->ids_stage, (size_t)max_M * max_k * sizeof(int32_t)) == cudaSuccess;
-    ok = ok && cudaMalloc(&c->lp_stage, (size_t)max_M * max_k * sizeof(float)) == cudaSuccess;
+    {
+        const size_t half = ((size_t)max_M * max_k * sizeof(int32_t) + 255) / 256 * 256;
+        void* dev_view = nullptr;
+        ok = ok && cudaHostAlloc(&c->res_host, 2 * half, cudaHostAllocMapped) == cudaSuccess;
+        ok = ok && cudaHostGetDevicePointer(&dev_view, c->res_host, 0) == cudaSuccess;
+        if (ok) {
+            c->ids_stage = reinterpret_cast<int32_t*>(dev_view);
+            c->lp_stage = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(dev_view) + half);
+            c->res_half = half;
+        }
+    }
     ok = ok && cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.err, 0, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.z, 0, z_elems * sizeof(float)) == cudaSuccess;
@@ -111,7 +124,8 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
     if (!c) return;
     cudaDeviceSynchronize();
     cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.smax); cudaFree(c->s.thr0); cudaFree(c->s.tickets); cudaFree(c->s.err);
-    cudaFree(c->s.logits); cudaFree(c->h_stage); cudaFree(c->ids_stage); cudaFree(c->lp_stage);
+    cudaFree(c->s.logits); cudaFree(c->h_stage);
+    if (c->res_host) cudaFreeHost(c->res_host);
     if (c->ev0) {
         for (int i = 0; i < kTimingEvents; ++i) { cudaEventDestroy(c->ev0[i]); cudaEventDestroy(c->ev1[i]); }
         delete[] c->ev0;
@@ -334,8 +348,8 @@ extern "C" int slimspec_head_topk_host(slimspec_ctx* c, const void* h_host, cons
     CK(cudaMemcpyAsync(c->h_stage, h_host, (size_t)M * d * sizeof(bf16), cudaMemcpyHostToDevice, st));
     int rc = slimspec_head_topk(c, c->h_stage, A, B, M, d, r, V, k, c->ids_stage, c->lp_stage, stream);
     if (rc != SLIMSPEC_OK) return rc;
-    CK(cudaMemcpyAsync(out_ids_host, c->ids_stage, (size_t)M * k * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    CK(cudaMemcpyAsync(out_logprobs_host, c->lp_stage, (size_t)M * k * sizeof(float), cudaMemcpyDeviceToHost, st));
-    CK(cudaStreamSynchronize(st));
+    CK(cudaStreamSynchronize(st));      // the kernels wrote the results into the mapped host buffer
+    memcpy(out_ids_host, c->res_host, (size_t)M * k * sizeof(int32_t));
+    memcpy(out_logprobs_host, reinterpret_cast<unsigned char*>(c->res_host) + c->res_half, (size_t)M * k * sizeof(float));
     return SLIMSPEC_OK;
 }
