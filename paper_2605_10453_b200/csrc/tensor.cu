@@ -5,10 +5,10 @@
 //   full-rank head   logits = h W X = h, W = W, same epilogue
 // (Section 4.1; the softmax of Section 3.2 and the candidate selection.)
 //
-// One CTA per SM, ten warps: warp 0 feeds a ring of shared-memory stages by TMA, one thread of
-// warp 1 issues the MMAs (128 rows x NV columns x 16 per instruction) into one of two
-// accumulator buffers in tensor memory, warps 2-9 read the finished buffer (a thread per row and
-// column half) and keep that row's running max / sum-exp / top-k while the next tile's MMAs run.
+// One CTA per SM: one warp feeds a ring of shared-memory stages by TMA, one thread of another
+// warp issues the MMAs (128 rows x NV columns x 16 per instruction) into one of two
+// accumulator buffers in tensor memory, eight epilogue warps read the finished buffer (a thread per
+// row and column half) and keep that row's running max / sum-exp / top-k while the next tile's MMAs run.
 #include "kernels.h"
 #include "ptx.cuh"
 #include <cuda.h>
@@ -19,7 +19,14 @@ namespace slimspec {
 
 static constexpr int kTcRows = 128;          // rows per tile = MMA M
 static constexpr int kTcKChunk = 64;         // K per stage: 64 bf16 = one 128-byte swizzle row
-static constexpr int kTcThreads = 320;       // TMA warp, MMA warp, eight epilogue warps
+// Twelve warps.  A warp reads only the lane quarter (warp id mod 4) of tensor memory and warps are
+// dealt to the SM's four schedulers by the same rule, so the rows of quarter q are worked on by the
+// scheduler q.  The thread that issues the MMAs loses its issue slots to busy epilogue warps of its
+// scheduler, so it (and the TMA thread) sit with the quarters that fill last: warp 2 loads, warp 3
+// issues, epilogue warps {0,4} {1,5} {6,10} {7,11} take quarters 0..3, warps 8 and 9 idle.  With up
+// to 64 rows in a tile neither special warp shares a scheduler with a busy warp.
+static constexpr int kTcThreads = 384;
+static constexpr int kTcLoadWarp = 2, kTcMmaWarp = 3;
 static constexpr int kTcMaxK = 32;           // largest k
 static constexpr int kTcList = 48;           // candidates a row parks before the list is compacted
 static constexpr int kTcListPitch = 49;      // words between two rows' lists in shared memory: odd, so lanes hit distinct banks
@@ -244,7 +251,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
         prefetch_tensor_map(&p.mapW);
         if (p.split) prefetch_tensor_map(&p.mapX2);
     }
-    if (warp == 1) tmem_alloc(&tmem_base_s, 2 * NV);
+    if (warp == kTcMmaWarp) tmem_alloc(&tmem_base_s, 2 * NV);
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -254,7 +261,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
     pdl_launch_dependents();
     pdl_wait();
 
-    if (warp == 0) {
+    if (warp == kTcLoadWarp) {
         // ================= producer: one thread issues the TMA loads =================
         if (lane == 0) {
             // ring positions are kept as (slot, phase) pairs: no division on this thread's path
@@ -290,7 +297,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == kTcMmaWarp) {
         // ================= MMA issuer =================
         // One thread feeds the tensor pipe, so its instruction count per K chunk is what bounds the
         // main loop once the data is there: descriptors are kept as a running low word (start
@@ -333,10 +340,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
                 if (alive) tc_commit(&acc_full[buf]);
             }
         }
-    } else {
+    } else if (warp != 8 && warp != 9) {
         // ================= epilogue: thread = row =================
         const int quarter = warp & 3;                        // the lane quarter this warp may read
-        const int half = (warp - 2) >> 2;                    // two warps share a quarter: each takes half the columns
+        const int half = (warp == 4 || warp == 5 || warp >= 10) ? 1 : 0;     // two warps share a quarter: each takes half the columns
+        const int slot = (quarter * 2 + half) * 32 + lane;  // 0..255 among the epilogue threads
         const int row = quarter * 32 + lane;
         const int m = rb * kTcRows + row;
         const bool live = m < p.M;
@@ -378,8 +386,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             // The lists live in local memory, which this kernel's small L1 hardly caches: a sort
             // there pays an L2 round trip per step.  Every MMA has completed by now (the last
             // accumulator was handed over), so the operand rings are dead: sort in that memory.
-            float* sv = reinterpret_cast<float*>(xarea) + (size_t)(tid - 64) * kTcListPitch;
-            int* si = reinterpret_cast<int*>(xarea + (size_t)kTcEpiThreads * kTcListPitch * 4) + (size_t)(tid - 64) * kTcListPitch;
+            float* sv = reinterpret_cast<float*>(xarea) + (size_t)slot * kTcListPitch;
+            int* si = reinterpret_cast<int*>(xarea + (size_t)kTcEpiThreads * kTcListPitch * 4) + (size_t)slot * kTcListPitch;
             for (int j = 0; j < cnt; ++j) {
                 sv[j] = cv[j];
                 si[j] = ci[j];
@@ -398,7 +406,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    if (warp == 1) tmem_dealloc(tmem_base, 2 * NV);
+    if (warp == kTcMmaWarp) tmem_dealloc(tmem_base, 2 * NV);
 }
 
 // ------------------------------------------------------------------------------------------
