@@ -139,6 +139,33 @@ def test_tensor_path_fullhead_and_planted_tie(ctx):
     assert ids[0, :2].tolist() == sorted([best, twin]) and lp[0, 0] == lp[0, 1]
 
 
+@pytest.mark.parametrize("M,k", [(6, 10), (140, 10), (70, 32)])
+def test_tensor_path_ascending_logits_fill_the_candidate_lists(ctx, M, k):
+    """Logits that grow with the column index: the bound taken from the first tiles prunes nothing,
+    nearly every later column is a candidate, so the per-row lists overflow and are compacted over
+    and over; runs of equal bf16 weights give ties that must resolve to the lower id."""
+    d, V = 64, 8 * 1400
+    g = torch.Generator().manual_seed(19)
+    h = (torch.rand((M, d), generator=g) * 0.5 + 0.25).to(torch.bfloat16)
+    s = torch.rand((d, 1), generator=g) * 0.2 + 0.05
+    W = (s * ((torch.arange(V, dtype=torch.float32) + 1.0) / V).view(1, V)).to(torch.bfloat16)
+    ref = oracle.fullhead_topk(oracle.bf16_bits(h), oracle.bf16_bits(W), k)
+    assert np.all(np.diff(ref["logits"], axis=1) >= 0)            # ascending, with ties
+    ctx.force_path(binding.PATH_TENSOR)
+    ids, lp = ctx.fullhead_topk(h.to(DEV), W.to(DEV), k)
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK and ctx.last_path() == binding.PATH_TENSOR
+    ids, lp = ids.cpu().numpy(), lp.cpu().numpy()
+    st = check_topk(ref, ids, lp)
+    assert st["max_lp_err"] <= 1e-3
+    # among equal logits the lower id comes first
+    for m in range(M):
+        for j in range(k - 1):
+            if lp[m, j] == lp[m, j + 1]:
+                assert ids[m, j] < ids[m, j + 1]
+    ctx.force_path(binding.PATH_AUTO)
+
+
 def test_stream_path_refuses_what_it_cannot_take(ctx):
     x = dev(synth.make_inputs(1, 64, 64, 8 * 100 + 4, seed=1))     # V not a multiple of 8
     ctx.force_path(binding.PATH_STREAM)
