@@ -490,6 +490,7 @@ __global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const He
     // ---- last CTA: merge the P slab records of every row, a few rows per round
     __threadfence();
     float* mrg = red;                                // the reduction and code areas are idle now
+    __shared__ float lse_s[32];                      // a row's log-sum-exp, by the row's place in the round
     uint32_t* stage_k = reinterpret_cast<uint32_t*>(ep_s);            // [rows][groups][32] keys, then ids
     const int row_words = P * RW;
     const int ngroups = (P + 31) >> 5;               // groups of 32 slabs, one warp each
@@ -526,18 +527,23 @@ __global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const He
             warp_topk_smem(reinterpret_cast<const uint32_t*>(rec + 2), reinterpret_cast<const int*>(rec + 2 + k),
                            s < P ? k : 0, k, stage_k + (size_t)job * 32, stage_i + (size_t)job * 32);
         }
-        __syncthreads();
-        // second level: a warp per row folds the groups' lists and finishes the log-softmax
-        if (warp < nrows) {
-            const int m = m0 + warp;
-            const float* rows = mrg + (size_t)warp * row_words;
+        // meanwhile the warps at the other end take the rows' log-sum-exp (it needs no list)
+        if (warp >= nwarps - nrows) {
+            const int rrow = nwarps - 1 - warp;
+            const float* rows = mrg + (size_t)rrow * row_words;
             float gm = -FLT_MAX;
             for (int s = lane; s < P; s += 32) gm = fmaxf(gm, rows[(size_t)s * RW]);
             gm = warp_max(gm);
             float gs = 0.f;
             for (int s = lane; s < P; s += 32) gs += rows[(size_t)s * RW + 1] * __expf(rows[(size_t)s * RW] - gm);
             gs = warp_sum(gs);
-            const float lse = gm + __logf(gs);
+            if (lane == 0) lse_s[rrow] = gm + __logf(gs);
+        }
+        __syncthreads();
+        // second level: a warp per row folds the groups' lists and finishes the log-softmax
+        if (warp < nrows) {
+            const int m = m0 + warp;
+            const float lse = lse_s[warp];
             const int lpl = 32 / ngroups;
             const int seg = (k + lpl - 1) / lpl;
             const int lw = lane / lpl, ls = lane - lw * lpl;
