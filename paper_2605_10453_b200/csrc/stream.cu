@@ -456,10 +456,17 @@ __global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const He
         for (int m = 0; m < MT; ++m) {
             if (!mine[m] || m >= p.M) continue;
             const float* rows = ep_s + (size_t)m * kMaxColWarps * 66;
-            float cm = -FLT_MAX;
-            for (int w = 0; w < NW; ++w) cm = fmaxf(cm, rows[w * 66]);
-            float cs = 0.f;
-            for (int w = 0; w < NW; ++w) cs += rows[w * 66 + 1] * __expf(rows[w * 66] - cm);
+            float cm = -FLT_MAX, cs = 0.f;
+            if (MT > 1 || NW > 4) {
+                // lane w takes warp w's (max, sum-exp); measured better than the loop except for one row
+                // with up to four warps
+                const float wm = lane < NW ? rows[lane * 66] : -FLT_MAX;
+                cm = warp_max(wm);
+                cs = warp_sum(lane < NW ? rows[lane * 66 + 1] * __expf(wm - cm) : 0.f);
+            } else {
+                for (int w = 0; w < NW; ++w) cm = fmaxf(cm, rows[w * 66]);
+                for (int w = 0; w < NW; ++w) cs += rows[w * 66 + 1] * __expf(rows[w * 66] - cm);
+            }
             const int first = ls * seg;
             const int len = (lw < NW && first < k) ? min(seg, k - first) : 0;
             const int lwc = lw < NW ? lw : 0;
