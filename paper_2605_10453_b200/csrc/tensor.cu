@@ -657,7 +657,10 @@ cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, in
         // A bound below each row's k-th largest logit, from the first sample tiles of the vocabulary:
         // it keeps the per-row candidate lists of the main pass almost idle.
         // (each sample tile yields two maxima per row, one per column half; k_tc_thr0 takes up to 64)
-        int nst = k > 16 ? 32 : 16;
+        // as many sample tiles as one wave of CTAs takes (the launch costs the same) and k_tc_thr0 reads
+        int nst = 32;
+        if (nst * p.nrb > sm_count) nst = sm_count / p.nrb;
+        if (nst < 1) nst = 1;
         if (nst > p.nct) nst = p.nct;
         if (2 * nst >= k && (size_t)2 * nst * p.nrb * kTcRows <= s.smax_elems) {
             TcParams q = p;
