@@ -366,11 +366,11 @@ def extra_points(torch, ctx, synth, binding, dev, peaks):
 
     out["slimspec_M1"] = point(1, 200)
     out["slimspec_M8"] = point(8, 100)
-    out["slimspec_M512"] = point(512, 5)
+    out["slimspec_M512"] = point(512, 20)
     del As, Bs
     # full-rank baseline: W is 1.05 GB, eight times the L2, so one copy is cold by itself
     Wd = synth.make_W(d, V, c1.seed).to(dev)
-    for M, n in ((1, 50), (8, 20), (512, 5)):
+    for M, n in ((1, 50), (8, 20), (512, 10)):
         h = synth.make_h(M, d, c1.seed).to(dev)
         ids = torch.empty((M, k), dtype=torch.int32, device=dev)
         lp = torch.empty((M, k), dtype=torch.float32, device=dev)
