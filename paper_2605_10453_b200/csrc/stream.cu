@@ -17,6 +17,13 @@ static constexpr int kMaxCtas = 256;         // slabs per row the merge can take
 static constexpr int kZChunkBytes = 64 * 1024;   // shared memory for the code, as (z, z) pairs
 static constexpr int kNoId = 0x7fffffff;
 
+// Bytes of the weight matrix (all CTAs together) the head kernel asks into the L2 while it waits
+// for the code: about what HBM delivers in that wait (measured; more only evicts what is needed).
+#ifndef SLIMSPEC_PF_MB
+#define SLIMSPEC_PF_MB 24
+#endif
+static constexpr size_t kPrefetchBytes = (size_t)SLIMSPEC_PF_MB << 20;
+
 struct HeadParams {
     const float* zT;      // [K][MT] fp32 code, transposed and zero-padded to MT rows
     const bf16* B;        // [K][V]
@@ -35,6 +42,7 @@ struct HeadParams {
     unsigned int* ticket;
     int* err;
     int wait_prev;        // 1: zT is written by the kernel launched just before (PDL)
+    int pf_rows;          // rows of the slab asked into the L2 while waiting for that kernel
 };
 
 // ------------------------------------------------------------------------------------------
@@ -281,7 +289,24 @@ __global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const He
     // the weights are on their way; let the next kernel in the stream come up behind this one,
     // then wait for the kernel that writes the code
     pdl_launch_dependents();
-    if (p.wait_prev) pdl_wait();
+    if (p.wait_prev) {
+        // Until the code is there this CTA can only wait, and while it waits HBM idles: ask the L2
+        // for the rows of the slab that come next (a hint; the loads of the main loop then hit the
+        // L2).  Launched early behind a kernel that still runs, the wait is several microseconds.
+        if (p.pf_rows > 0 && npass > 0) {
+            const int pun0 = min(units_per_pass, my_units);
+            const int lines = (pun0 * 16 + 127) / 128 + 1;          // the slab's row segment need not start on a line
+            const int r0 = min(K, stepU), r1 = min(K, stepU + p.pf_rows);
+            const char* seg = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
+            const size_t row_bytes = (size_t)V * sizeof(bf16);
+            const int last = pun0 * 16 - 1;                          // last byte of the row segment
+            for (int i = tid; i < (r1 - r0) * lines; i += blockDim.x) {
+                const int r = r0 + i / lines, l = i - (i / lines) * lines;
+                prefetch_l2(seg + (size_t)r * row_bytes + min(l * 128, last));
+            }
+        }
+        pdl_wait();
+    }
 
     float run_max[MT], run_sum[MT];
     uint32_t lst_k[MT];                              // lane j < k: key of the j-th best so far
@@ -710,6 +735,11 @@ cudaError_t stream_head(const float* zT, const bf16* B, int M, int mt, int K, in
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     hp.wait_prev = after_producer_kernel ? 1 : 0;
+    {
+        const size_t row_bytes = (size_t)g.pass_units * 16 * g.ncta;      // one row of every slab's first pass
+        const size_t rows = row_bytes ? kPrefetchBytes / row_bytes : 0;
+        hp.pf_rows = after_producer_kernel ? (int)(rows < (size_t)K ? rows : (size_t)K) : 0;
+    }
     switch (mt) {
     case 1: return launch_head<1, 16>(hp, g, after_producer_kernel, st);
     case 2: return launch_head<2, 16>(hp, g, after_producer_kernel, st);
