@@ -75,6 +75,20 @@ def head_flops(M, d, r, V):
     return 2 * M * (d * r + r * V)
 
 
+def fullhead_bytes(M, d, V, k):
+    """Algorithmic bytes of one full-rank call: W and h read once, top-k written."""
+    return 2 * d * V + 2 * M * d + 8 * M * k
+
+
+def fullhead_flops(M, d, V):
+    return 2 * M * d * V
+
+
+def bytes_ratio_target(d, r, V):
+    """The speed-up over the full-rank head the low-rank head should reach: 0.8 of the ratio of weights read."""
+    return 0.8 * (d * V) / (d * r + r * V)
+
+
 # --------------------------------------------------------------------------- clocks
 
 class ClockSampler:

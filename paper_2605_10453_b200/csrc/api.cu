@@ -34,7 +34,7 @@ static const int kTimingEvents = 256;
 
 static const int kMaxParts = 256;      // most V slabs any kernel writes per row
 static const int kStreamMaxRows = 4;   // largest M the streaming path is chosen for
-static const int kSplitCodeRows = 64;   // tensor path: z carried as hi + lo bf16 parts up to this many rows
+static const int kSplitCodeRows = 256;  // tensor path: z carried as hi + lo bf16 parts while the call is HBM-bound (up to this many rows)
 static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }

@@ -382,3 +382,90 @@ def test_back_to_back_calls_keep_stream_order(ctx, M):
         ids, lp = alone[i % 2]
         assert torch.equal(out_ids[i], ids), "call %d" % i
         assert torch.equal(out_lp[i], lp), "call %d" % i
+
+
+# ---------------------------------------------------------------- large batches: oracle on sampled rows
+
+def sampled_rows(M, extra=8, seed=0):
+    """Rows at every position class of a 128-row tile, the ends, the middle, plus seeded extras."""
+    rng = np.random.default_rng(seed)
+    base = {0, 1, 63, 64, 127, 128, M // 2, M - 2, M - 1}
+    return sorted({m for m in base if 0 <= m < M} | set(rng.integers(0, M, extra).tolist()))
+
+
+@pytest.fixture(scope="module")
+def big_ctx():
+    c = binding.Context(max_M=1024, max_d=8192, max_V=160000, max_k=16)
+    yield c
+    c.close()
+
+
+def test_fullhead_throughput_batch_sampled_rows(big_ctx):
+    """The standard head at the throughput batch (M = 512, d = 4096): K is too long for a resident
+    row block, so the activations go through their own ring next to the weight ring."""
+    c = synth.CONFIGS["c3"]
+    M = 512
+    h = synth.make_h(M, c.d, c.seed)
+    W = synth.make_W(c.d, c.V, c.seed)
+    big_ctx.force_path(binding.PATH_AUTO)
+    ids, lp = big_ctx.fullhead_topk(h.to(DEV), W.to(DEV), c.k)
+    torch.cuda.synchronize()
+    assert big_ctx.last_error() == binding.OK and big_ctx.last_path() == binding.PATH_TENSOR
+    rows = sampled_rows(M)
+    ref = oracle.fullhead_topk(oracle.bf16_bits(h)[rows], oracle.bf16_bits(W), c.k)
+    st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy(), rows=rows)
+    assert st["max_lp_err"] <= 1e-3        # h is exact in bf16: only fp32 accumulation differs
+
+
+@pytest.mark.parametrize("r,M", [(2048, 256), (512, 1024), (512, 256)])
+def test_sweep_large_batches_sampled_rows(big_ctx, r, M):
+    """d = 8192 heads of the rank sweep with several row blocks."""
+    d, V, k = synth.SWEEP_D, synth.SWEEP_V, 10
+    x = synth.make_inputs(M, d, r, V, seed=7)
+    g = dev(x)
+    big_ctx.force_path(binding.PATH_AUTO)
+    ids, lp = big_ctx.slimspec_head_topk(g["h"], g["A"], g["B"], k)
+    torch.cuda.synchronize()
+    assert big_ctx.last_error() == binding.OK and big_ctx.last_path() == binding.PATH_TENSOR
+    rows = sampled_rows(M, extra=4)
+    b = obits(x)
+    ref = oracle.head_topk(b["h"][rows], b["A"], b["B"], k)
+    st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy(), rows=rows)
+    assert st["max_lp_err"] <= LOGPROB_TOL
+
+
+def test_sweep_fullhead_largest_batch_sampled_rows(big_ctx):
+    """Full rank at d = 8192, M = 1024: eight row blocks, 128 K chunks per tile."""
+    d, V, k, M = synth.SWEEP_D, synth.SWEEP_V, 10, 1024
+    h = synth.make_h(M, d, 7)
+    W = synth.make_W(d, V, 7)
+    big_ctx.force_path(binding.PATH_AUTO)
+    ids, lp = big_ctx.fullhead_topk(h.to(DEV), W.to(DEV), k)
+    torch.cuda.synchronize()
+    assert big_ctx.last_error() == binding.OK and big_ctx.last_path() == binding.PATH_TENSOR
+    rows = sampled_rows(M, extra=2)
+    ref = oracle.fullhead_topk(oracle.bf16_bits(h)[rows], oracle.bf16_bits(W), k)
+    st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy(), rows=rows)
+    assert st["max_lp_err"] <= 2e-3
+
+
+@pytest.mark.parametrize("M", [16, 128])
+def test_sharpened_logits_keep_the_logit_bound(big_ctx, M):
+    """Logits scaled by four (the larger-vocabulary workload) at batch sizes where the code z is a
+    tensor-core operand: raw logits must still lie within 2e-2 of the oracle's, which a code
+    rounded once to bf16 would miss."""
+    c = synth.CONFIGS["c2"]
+    x = synth.make_inputs(M, c.d, c.r, c.V, seed=c.seed, logit_scale=c.logit_scale)
+    g = dev(x)
+    big_ctx.force_path(binding.PATH_AUTO)
+    out = big_ctx.slimspec_head_logits(g["h"], g["A"], g["B"])
+    ids, lp = big_ctx.slimspec_head_topk(g["h"], g["A"], g["B"], c.k)
+    torch.cuda.synchronize()
+    assert big_ctx.last_error() == binding.OK
+    rows = sampled_rows(M, extra=2)
+    b = obits(x)
+    ref = oracle.head_topk(b["h"][rows], b["A"], b["B"], c.k)
+    err = np.max(np.abs(out.cpu().numpy()[rows].astype(np.float64) - ref["logits"]))
+    assert err <= 2e-2, "logit error %.3e" % err
+    st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy(), rows=rows)
+    assert st["max_lp_err"] <= LOGPROB_TOL

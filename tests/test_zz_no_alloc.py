@@ -46,6 +46,21 @@ def test_static_scratch_entry_point_matches_context_entry_point_twice():
     ctx.close()
 
 
+def test_static_scratch_entry_point_matches_the_oracle():
+    """The same entry point against the CPU oracle (not only against the context-based call)."""
+    import oracle
+    from parity import check_topk
+    M, d, r, V, k = 3, 512, 128, 8 * 1501, 7
+    x = synth.make_inputs(M, d, r, V, seed=13)
+    g = {n: t.to(DEV) for n, t in x.items()}
+    b = {n: oracle.bf16_bits(t) for n, t in x.items()}
+    ref = oracle.head_topk(b["h"], b["A"], b["B"], k)
+    for _ in range(2):
+        ids, lp = _static(g, k)
+        st = check_topk(ref, ids, lp)
+        assert st["max_lp_err"] <= 1e-3
+
+
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
     lib = binding.load()
     g = {n: t.to(DEV) for n, t in synth.make_inputs(2, 64, 64, 800, seed=1).items()}
