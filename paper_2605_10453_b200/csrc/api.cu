@@ -32,10 +32,11 @@ struct slimspec_ctx {
 };
 static const int kTimingEvents = 256;
 
-static const int kMaxParts = 256;      // most V slabs any kernel writes per row
-static const int kStreamMaxRows = 4;   // largest M the streaming path is chosen for
+static const int kMaxParts = 320;      // most split-V records any kernel writes per row
+static const int kStreamMaxRows = 16;  // largest M the streaming path is chosen for
 static const int kSplitCodeRows = 256;  // tensor path: z carried as hi + lo bf16 parts while the call is HBM-bound (up to this many rows)
-static const int kRowPad = 8;          // the streaming kernels read z in tiles of up to 8 rows
+static const int kRowPad = 8;          // rows of the generic path's fp32 code are padded to this
+static const int kStreamTile = 16;     // rows one launch of the streaming kernels takes
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
@@ -72,11 +73,11 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     c->s.max_parts = kMaxParts;
     const size_t mpad = (size_t)round_up(max_M, kRowPad);
     const size_t z_elems = mpad * (size_t)max_d;
-    // split-V records, padded to 16 bytes: the streaming path writes <= 8 rows x 256 slabs, the
+    // split-V records, padded to 16 bytes: the streaming path writes <= 16 rows x 320 records, the
     // tensor path 128 * nrb rows x (SMs / nrb) slabs
     const int rec_k = max_k < 32 ? max_k : 32;
     const size_t mpad128 = (size_t)round_up(max_M, 128);
-    const size_t part_elems = ((size_t)kRowPad * 256 + (size_t)(c->sm_count + 12) * 256 + 2 * mpad128) *
+    const size_t part_elems = ((size_t)kStreamTile * kMaxParts + (size_t)(c->sm_count + 12) * 256 + 2 * mpad128) *
                               (size_t)round_up(2 + 2 * rec_k, 4);
     // K-split partial tiles of the tensor-core down-projection: one 128 x 128 fp32 tile per SM, or one split
     size_t zpart_elems = (size_t)(c->sm_count + 12) * 128 * 128;
@@ -84,6 +85,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     bool ok = true;
     ok = ok && cudaMalloc(&c->s.z, z_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.zfrag, stream_code_bytes(max_d)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zb, 2 * mpad128 * (size_t)max_d * sizeof(bf16)) == cudaSuccess;
     if (ok) c->s.zb_lo = c->s.zb + mpad128 * (size_t)max_d;
@@ -109,6 +111,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     ok = ok && cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.err, 0, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.z, 0, z_elems * sizeof(float)) == cudaSuccess;
+    ok = ok && stream_prepare() == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -123,7 +126,7 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
 {
     if (!c) return;
     cudaDeviceSynchronize();
-    cudaFree(c->s.z); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.smax); cudaFree(c->s.thr0); cudaFree(c->s.tickets); cudaFree(c->s.err);
+    cudaFree(c->s.z); cudaFree(c->s.zfrag); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.smax); cudaFree(c->s.thr0); cudaFree(c->s.tickets); cudaFree(c->s.err);
     cudaFree(c->s.logits); cudaFree(c->h_stage);
     if (c->res_host) cudaFreeHost(c->res_host);
     if (c->ev0) {
@@ -243,8 +246,8 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
     int path = c->forced_path;
     const bool ptr_ok = aligned16(h) && aligned16(Bm) && (!lowrank || aligned16(A)) &&
                         (mode == 0 || aligned16(logits));
-    StreamPlan sp = stream_plan(M, d, K, V, mode == 0 ? k : 1, c->sm_count);
-    const bool stream_ok = sp.ok && ptr_ok && (!lowrank || r % 16 == 0);
+    StreamPlan sp = stream_plan(M, K, V, mode == 0 ? k : 1, c->sm_count);
+    const bool stream_ok = sp.ok && ptr_ok && d % 2 == 0 && (!lowrank || r % 16 == 0);
     const bool tensor_fits = tensor_ok(M, K, V, k, mode) && ptr_ok && (!lowrank || (d % 64 == 0 && r >= 64));
     if (path == SLIMSPEC_PATH_AUTO) {
         // FP32 FMAs keep up with HBM only for a few rows; beyond that the tensor cores take over
@@ -291,13 +294,13 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         return SLIMSPEC_OK;
     }
 
-    // streaming path: row tiles of up to 8 rows, each streams the K x V matrix once
-    for (int m0 = 0; m0 < M; m0 += 8) {
-        const int mrows = (M - m0 < 8) ? (M - m0) : 8;
-        StreamPlan p = stream_plan(mrows, d, K, V, mode == 0 ? k : 1, c->sm_count);
+    // streaming path: row tiles of up to 16 rows, each streams the K x V matrix once
+    for (int m0 = 0; m0 < M; m0 += kStreamTile) {
+        const int mrows = (M - m0 < kStreamTile) ? (M - m0) : kStreamTile;
         const bf16* hm = h + (size_t)m0 * d;
-        if (lowrank) CK(stream_downproj(hm, A, mrows, p.mt, d, r, c->s, st));
-        else CK(stream_widen_t(hm, mrows, p.mt, d, c->s.z, st));
+        const int kk = mode == 0 ? k : 1;
+        if (lowrank) CK(stream_code(hm, A, mrows, d, r, V, kk, c->s.zfrag, c->sm_count, st));
+        else CK(stream_widen(hm, mrows, d, V, kk, c->s.zfrag, c->sm_count, st));
         int slot = -1;
         if (c->timing_on) {
             if (c->timing_used == kTimingEvents) { int rc = timing_drain(c); if (rc != SLIMSPEC_OK) return rc; }
@@ -305,7 +308,7 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
             CK(cudaEventRecord(c->ev0[slot], st));
         }
         // an event between the two kernels serialises them: the timed kernel then runs alone
-        CK(stream_head(c->s.z, Bm, mrows, p.mt, K, V, k, mode,
+        CK(stream_head(c->s.zfrag, lowrank, Bm, mrows, K, V, kk, mode,
                        mode == 0 ? ids + (size_t)m0 * k : nullptr,
                        mode == 0 ? logprobs + (size_t)m0 * k : nullptr,
                        mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, slot < 0, st));

@@ -13,7 +13,8 @@ typedef __nv_bfloat16 bf16;
 // slab's k best (logit, id) pairs in (logit desc, id asc) order.
 // Layout in the context's scratch: float pm[P], ps[P], pv[P][k]; int pi[P][k] per row.
 struct Scratch {
-    float* z;            // fp32 code (or widened h); generic path [M][K], streaming path transposed [K][mt]
+    float* z;            // fp32 code (or widened h) of the generic path, [M][K]
+    uint32_t* zfrag;     // streaming path: the code, as fp32 or as tensor-core fragments (see stream.cu)
     bf16* zb;            // bf16 code [M][r] for the tensor-core path
     bf16* zb_lo;         // its rounding remainder (z - zb), bf16: used while the call is HBM-bound
     float* zpart;        // K-split partial tiles of the tensor-core down-projection
@@ -40,18 +41,24 @@ cudaError_t generic_softmax_topk(const float* logits, int M, int V, int k, int32
 // ---- streaming path (small M) -------------------------------------------------------
 struct StreamPlan {
     int ok;          // 0: shapes not supported by the streaming kernels
-    int mt;          // rows per launch (1, 2, 4, 8)
+    int mt;          // rows the kernel keeps per launch (8 or 16)
     int ncta;        // V slabs = CTAs
-    int launches;    // kernels per call (for the launch counter)
+    int parts;       // records per row the head kernel writes (slabs x column passes)
+    int launches;    // kernels per row tile (for the launch counter)
 };
-StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count);
-// z^T = (h A)^T for M <= 8 rows, rows M..mt-1 zero-filled; r must be a multiple of 16.
-cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
-                            cudaStream_t st);
-// z^T = widened h^T (full-rank head: no down-projection).
-cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st);
-// logits = z B streamed once; mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
-cudaError_t stream_head(const float* z, const bf16* B, int M, int mt, int K, int V, int k, int mode,
+// Once per device, before the first launch: loads the kernels and sets their shared-memory limits.
+cudaError_t stream_prepare();
+// K: contraction length of the streamed matrix (r, or d for the full-rank head).
+StreamPlan stream_plan(int M, int K, int V, int k, int sm_count);
+// Bytes of the code fragments for a streamed matrix of K rows (two parts: value and remainder).
+size_t stream_code_bytes(int K);
+// code = h A for M <= 16 rows, in the form the head kernel for these shapes reads; d even, r a multiple of 16.
+cudaError_t stream_code(const bf16* h, const bf16* A, int M, int d, int r, int V, int k, uint32_t* code, int sm_count,
+                        cudaStream_t st);
+// code = h itself (full-rank head: no down-projection).
+cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* code, int sm_count, cudaStream_t st);
+// logits = z B streamed once (M <= 16); mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
+cudaError_t stream_head(const uint32_t* code, bool lowrank, const bf16* B, int M, int K, int V, int k, int mode,
                         int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
                         bool after_producer_kernel, cudaStream_t st);
 

@@ -17,10 +17,11 @@ using namespace slimspec;
 namespace {
 
 // Layout of the static scratch, in bytes.  Limits: M <= 8 rows, r <= SLIMSPEC_STATIC_MAX_R,
-// k <= 32, at most 256 V slabs (one per SM).
-constexpr size_t kZBytes = (size_t)SLIMSPEC_STATIC_MAX_R * 8 * sizeof(float);       // z^T [r][8]
+// k <= 32, at most 320 split-V records per row.
+constexpr size_t kZBytes = (size_t)(SLIMSPEC_STATIC_MAX_R / 16) * 2 * 512 + 1024;   // the code, in its largest form
 constexpr size_t kRecWords = 68;                                                     // 2 + 2*32, padded to 4
-constexpr size_t kPartBytes = (size_t)8 * 256 * kRecWords * sizeof(float);           // [8 rows][256 slabs]
+constexpr int kStaticParts = 320;
+constexpr size_t kPartBytes = (size_t)8 * kStaticParts * kRecWords * sizeof(float);  // [8 rows][320 records]
 constexpr size_t kCtlBytes = 256;                                                    // ticket, error word
 constexpr size_t kScratchBytes = kZBytes + kPartBytes + kCtlBytes;
 
@@ -48,6 +49,8 @@ int setup_current_device(DeviceSetup** out)
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
+        // load the kernels now, so that no later call has to (loading a module allocates)
+        if (stream_prepare() != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         s.base = static_cast<unsigned char*>(ptr);
         s.sm_count = sms;
         s.ready = true;
@@ -70,21 +73,21 @@ extern "C" int slimspec_head_topk_static(const void* h, const void* A, const voi
     DeviceSetup* dev = nullptr;
     int rc = setup_current_device(&dev);
     if (rc != SLIMSPEC_OK) return rc;
-    StreamPlan plan = stream_plan(M, d, r, V, k, dev->sm_count);
-    if (!plan.ok || r % 16 != 0 || !aligned16(h) || !aligned16(A) || !aligned16(B)) return SLIMSPEC_ERR_ALIGN;
-    if (plan.ncta > 256) return SLIMSPEC_ERR_STATIC_LIMIT;
+    StreamPlan plan = stream_plan(M, r, V, k, dev->sm_count);
+    if (!plan.ok || r % 16 != 0 || d % 2 != 0 || !aligned16(h) || !aligned16(A) || !aligned16(B)) return SLIMSPEC_ERR_ALIGN;
+    if (plan.parts > kStaticParts) return SLIMSPEC_ERR_STATIC_LIMIT;
 
     Scratch s = {};
-    s.z = reinterpret_cast<float*>(dev->base);
+    s.zfrag = reinterpret_cast<uint32_t*>(dev->base);
     s.part = reinterpret_cast<float*>(dev->base + kZBytes);
     s.tickets = reinterpret_cast<unsigned int*>(dev->base + kZBytes + kPartBytes);
     s.err = reinterpret_cast<int*>(dev->base + kZBytes + kPartBytes + 128);
-    s.max_parts = 256;
+    s.max_parts = kStaticParts;
     cudaStream_t st = (cudaStream_t)stream;
     // The array keeps whatever the last call left; the ticket and the error word must start at 0.
     if (cudaMemsetAsync(dev->base + kZBytes + kPartBytes, 0, kCtlBytes, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
-    if (stream_downproj((const bf16*)h, (const bf16*)A, M, plan.mt, d, r, s, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
-    if (stream_head(s.z, (const bf16*)B, M, plan.mt, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, st) !=
+    if (stream_code((const bf16*)h, (const bf16*)A, M, d, r, V, k, s.zfrag, dev->sm_count, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
+    if (stream_head(s.zfrag, true, (const bf16*)B, M, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, st) !=
         cudaSuccess) {
         cudaGetLastError();
         return SLIMSPEC_ERR_CUDA;

@@ -1,349 +1,777 @@
-// Streaming path for small M (<= 8 rows per launch): the K x V weight matrix is read from HBM
-// exactly once, in split-V slabs (one CTA per SM), with coalesced 128-bit loads held in flight
-// in registers and consumed by packed FP32 FMAs.
-// The logits never leave the SM: each CTA keeps a running max / sum-exp / top-k per row and
-// the last CTA to finish merges the per-slab records (Section 4.1 up-projection, the
-// softmax of Section 3.2 in online form, and the candidate selection).
+// Streaming path for small M (up to 16 rows per launch): the K x V weight matrix is read from HBM
+// exactly once, in split-V slabs (one CTA per SM), every warp instruction fetching 512 contiguous
+// bytes of one row.  The logits never leave the SM: every CTA keeps max / sum-exp / top-k per
+// row for its slab, and the last CTA to finish merges the per-slab records (Section 4.1
+// up-projection, the softmax of Section 3.2 in online form, and the candidate selection).
+//
+// Two main loops feed one epilogue:
+//   k_stream_head_fma  one or two rows: loads held in flight in registers, packed FP32 FMAs
+//                      against the fp32 code;
+//   k_stream_head_mma  three to sixteen rows: a cp.async ring in shared memory, ldmatrix and
+//                      warp-level tensor-core instructions (mma.sync m16n8k16, bf16 in, fp32
+//                      accumulate) with the rows of the batch on the instruction's 16-row side and
+//                      the code as bf16 value + bf16 remainder.  (On this GPU one such instruction
+//                      holds the SM's legacy tensor pipe for 8 cycles: 8 of them per 2 KB of
+//                      weights keep up with HBM, 16 do not -- hence the packed fragments below.)
+// The code itself comes from k_stream_code: the same fragment scheme applied to h A, split over
+// K across the CTAs of a cluster and folded through distributed shared memory.
 #include "kernels.h"
 #include "ptx.cuh"
 #include <float.h>
-#include <type_traits>
+#include <string.h>
 
 namespace slimspec {
 
-static constexpr int kMaxColThreads = 256;   // threads across one pass's columns, 8 columns each
-static constexpr int kMaxColWarps = kMaxColThreads / 32;
-static constexpr int kMaxCtas = 256;         // slabs per row the merge can take
-static constexpr int kZChunkBytes = 64 * 1024;   // shared memory for the code, as (z, z) pairs
+static constexpr int kHeadWarps = 14;                 // warps of a head CTA: 64 columns each per pass
+static constexpr int kHeadThreads = kHeadWarps * 32;
+static constexpr int kMaxStages = 8;                  // most stages of the shared-memory ring
+static constexpr int kCand = 256;                     // candidates one row may park in a CTA's epilogue
+static constexpr int kMergeCand = 128;                // candidates one row may park in the final merge
+static constexpr int kMergeLists = 10;                // slab records a lane owns in the final merge
+static constexpr int kMaxRecords = 32 * kMergeLists;  // records per row the merge can take
 static constexpr int kNoId = 0x7fffffff;
+enum : int { kCodeF32 = 0, kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3 };
+static constexpr size_t kZOneChunkBytes = 48 * 1024;  // code fragments up to this size stay whole in shared memory
+static constexpr size_t kZChunkBytes = 32 * 1024;     // else they pass through two buffers of this size
+static constexpr int kEpFixedBytes = 64 + (16 * 64 + 16 + 16 + 16 + 16 * 16) * 4;
+static constexpr int kFmaLoads = 16;                  // 16-byte loads a thread of the FMA kernel keeps in flight
+static constexpr size_t kFmaCodeBytes = 64 * 1024;    // most shared memory the FMA kernel spends on the code
 
 // Bytes of the weight matrix (all CTAs together) the head kernel asks into the L2 while it waits
 // for the code: about what HBM delivers in that wait (measured; more only evicts what is needed).
 #ifndef SLIMSPEC_PF_MB
-#define SLIMSPEC_PF_MB 24
+#define SLIMSPEC_PF_MB 40
 #endif
 static constexpr size_t kPrefetchBytes = (size_t)SLIMSPEC_PF_MB << 20;
 
 struct HeadParams {
-    const float* zT;      // [K][MT] fp32 code, transposed and zero-padded to MT rows
-    const bf16* B;        // [K][V]
+    const uint32_t* zfrag;    // code: fragments [nkb][ZP][32 lanes][4 words], or fp32 [K][2] for the FMA kernel
+    const bf16* B;            // [K][V]
     int M, K, V, k, mode;
-    int ncta;             // slabs
-    int units_base, units_rem;   // V/8 column units: slab c has units_base + (c < units_rem)
-    int pass_units;       // most units one pass covers (<= ct)
-    int ct, rg;           // column threads (multiple of 32) and row groups: blockDim = ct * rg
-    int kc;               // rows of the code per shared-memory chunk (K, or a multiple of rg * U)
-    int rec_words;        // words per split-V record: max, sum-exp, k keys, k ids, padded to 4
-    int merge_rows;       // rows the last CTA merges per round
+    int ncta;                 // slabs
+    int units_base, units_rem;    // V/8 column units: slab c has units_base + (c < units_rem)
+    int pitch_units;          // 16-byte units between two rows of a stage (odd, >= the widest slab)
+    int ns;                   // stages of the ring
+    int nkb;                  // 16-row blocks of the matrix: ceil(K / 16)
+    int kb_chunk, nchunks;    // blocks of code fragments per shared-memory chunk, chunks
+    unsigned int zarea_bytes; // shared memory the code takes
+    int ct, rg;               // FMA kernel: column threads (one per unit of the widest slab) and row groups
+    int rec_words;            // words per record: max, sum-exp, k (key, id) pairs, padded to 4
     int32_t* ids;
     float* logprobs;
     float* logits;
-    float* part;          // split-V records [M][ncta][rec_words]
+    float* part;              // records [M][ncta * npass][rec_words]
     unsigned int* ticket;
     int* err;
-    int wait_prev;        // 1: zT is written by the kernel launched just before (PDL)
-    int pf_rows;          // rows of the slab asked into the L2 while waiting for that kernel
+    int wait_prev;            // 1: the code is written by the kernel launched just before (PDL)
+    int pf_rows;              // rows of the slab asked into the L2 before that kernel is waited for
 };
 
 // ------------------------------------------------------------------------------------------
-// Selection.  Candidates are (key, id) with key = f2key(logit) and key 0 = none; the order is
-// (key descending, id ascending).  Every lane offers the head of a list that is already in that
-// order; each round takes the best head of the warp and advances that lane's list.  Lane j < k
-// ends up with the j-th best.
+// Small PTX helpers of this file.
 
-// One round: does this lane's head win?  The winner has the largest key, and among equal keys
-// the lowest id (the second reduction runs only when keys tie).  With no candidate left the
-// "winner" is an empty entry (key 0, id kNoId).
-__device__ __forceinline__ bool round_winner(uint32_t hk, int hi)
+// Streaming load of weights: not kept in the L1, and first in line for eviction from the L2, so
+// that the stream does not push out what is meant to stay there (the rows of the next call's
+// matrices asked for ahead of time, the down-projection matrix, the code).
+__device__ __forceinline__ uint64_t policy_evict_first()
 {
-    const uint32_t wk = warp_max_u32(hk);
-    bool win = hk == wk;
-    const unsigned tied = __ballot_sync(0xffffffffu, win);
-    if (tied & (tied - 1)) {
-        const uint32_t wi = warp_min_u32(win ? (uint32_t)hi : 0xffffffffu);
-        win = win && (uint32_t)hi == wi;
-    }
-    return win;
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint4 ldg_stream(const void* p, uint64_t pol)
+{
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p), "l"(pol));
+    return r;
+}
+__device__ __forceinline__ void prefetch_l2_keep(const void* p) { asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p)); }
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
 }
 
-// The winner of round j drops its head into out_k[j], out_i[j] (shared memory, one pair of
-// 32-entry arrays per warp), so nothing but the pop of the winner's list sits between two
-// rounds, and that pop is a select, not a branch.
-
-// Lists held in registers, NL entries per lane (unused entries: key 0, id kNoId).
-template <int NL>
-__device__ __forceinline__ void warp_topk_regs(uint32_t (&ck)[NL], int (&ci)[NL], int k, uint32_t* out_k, int* out_i)
+// D (16 x 8, fp32) += A (16 x 16, bf16, row-major fragment) * B (16 x 8, bf16, column fragment)
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint4& a, uint32_t b0, uint32_t b1)
 {
-    for (int j = 0; j < k; ++j) {
-        const bool win = round_winner(ck[0], ci[0]);
-        if (win) { out_k[j] = ck[0]; out_i[j] = ci[0]; }
-#pragma unroll
-        for (int s = 0; s + 1 < NL; ++s) { ck[s] = win ? ck[s + 1] : ck[s]; ci[s] = win ? ci[s + 1] : ci[s]; }
-        ck[NL - 1] = win ? 0u : ck[NL - 1];
-        ci[NL - 1] = win ? kNoId : ci[NL - 1];
-    }
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
 }
 
-// Lists held in shared memory: this lane's list is keys[0..len), ids[0..len).  The entry after
-// the head is fetched ahead, so a pop never waits for shared memory.
-__device__ __forceinline__ void warp_topk_smem(const uint32_t* keys, const int* ids, int len, int k, uint32_t* out_k,
-                                               int* out_i)
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src)
 {
-    int pos = 0;
-    uint32_t hk = len > 0 ? keys[0] : 0u;
-    int hi = len > 0 ? ids[0] : kNoId;
-    uint32_t nk = len > 1 ? keys[1] : 0u;
-    int ni = len > 1 ? ids[1] : kNoId;
-    for (int j = 0; j < k; ++j) {
-        const bool win = round_winner(hk, hi);
-        if (win) { out_k[j] = hk; out_i[j] = hi; }
-        pos += win ? 1 : 0;
-        hk = win ? nk : hk;
-        hi = win ? ni : hi;
-        const bool more = pos + 1 < len;
-        const int nx = more ? pos + 1 : 0;
-        const uint32_t tk = keys[len > 0 ? nx : 0];
-        const int ti = ids[len > 0 ? nx : 0];
-        nk = more ? tk : 0u;
-        ni = more ? ti : kNoId;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst_smem)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// wait until at most n of this thread's committed groups are still in flight
+__device__ __forceinline__ void cp_async_wait_pending(int n)
+{
+    switch (n) {
+    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+    case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+    case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
     }
 }
 
-// compare-exchange so that (ka, ia) comes before (kb, ib)
-__device__ __forceinline__ void order2(uint32_t& ka, int& ia, uint32_t& kb, int& ib)
+// four 8 x 8 bf16 matrices from shared memory, transposed on the way: lane l supplies the address
+// of row (l & 7) of matrix (l >> 3); register i of lane (g, t) receives rows 2t, 2t+1 of column g
+// of matrix i
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3, uint32_t addr)
 {
-    const bool swap = (ka < kb) || (ka == kb && ia > ib);
-    const uint32_t tk = swap ? kb : ka;
-    const int ti = swap ? ib : ia;
-    kb = swap ? ka : kb;
-    ib = swap ? ia : ib;
-    ka = tk;
-    ia = ti;
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
 }
 
-// sort the first 8 candidates of a 9-entry list (19 compare-exchanges)
-__device__ __forceinline__ void sort8(uint32_t (&k)[9], int (&i)[9])
+// Arrival counter with release / acquire semantics at GPU scope: what the CTA wrote before its
+// barrier is visible to whoever reads the counter's later values.
+__device__ __forceinline__ unsigned int ticket_take(unsigned int* ticket)
 {
-#define SLIMSPEC_CE(a, b) order2(k[a], i[a], k[b], i[b])
-    SLIMSPEC_CE(0, 1); SLIMSPEC_CE(2, 3); SLIMSPEC_CE(4, 5); SLIMSPEC_CE(6, 7);
-    SLIMSPEC_CE(0, 2); SLIMSPEC_CE(1, 3); SLIMSPEC_CE(4, 6); SLIMSPEC_CE(5, 7);
-    SLIMSPEC_CE(1, 2); SLIMSPEC_CE(5, 6); SLIMSPEC_CE(0, 4); SLIMSPEC_CE(3, 7);
-    SLIMSPEC_CE(1, 5); SLIMSPEC_CE(2, 6);
-    SLIMSPEC_CE(1, 4); SLIMSPEC_CE(3, 6);
-    SLIMSPEC_CE(2, 4); SLIMSPEC_CE(3, 5);
-    SLIMSPEC_CE(3, 4);
-#undef SLIMSPEC_CE
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(ticket) : "memory");
+    return old;
 }
 
 // ------------------------------------------------------------------------------------------
-// z^T = (h A)^T for M <= MT rows.  A CTA owns 16 columns of A (two 16-byte units) over all d
-// rows, so no partial sums cross CTAs; a thread owns one unit and every (NT/2)-th row, with
-// RB row loads in flight at a time.  Rows M..MT-1 of z^T are written as zeros.
-template <int MT, int NT, int RB>
-__global__ void __launch_bounds__(NT) k_stream_downproj(const bf16* __restrict__ h, const bf16* __restrict__ A, int M,
-                                                         int d, int r, float* __restrict__ zT)
+// Selection.  Candidates are (key, id) with key = f2key(logit) and key 0 = none; the order is
+// (key descending, id ascending).
+
+// The k-th largest (k = 1..32) of the warp's 32 lane values, by counting: a lane's rank is the
+// number of lanes ahead of it (larger key, or equal key and lower lane).
+__device__ __forceinline__ uint32_t warp_kth_largest(uint32_t key, int k, int lane)
 {
-    pdl_launch_dependents();
-    __shared__ float red[NT / 32][MT][16];
-    const int t = threadIdx.x, u = t & 1, rl = t >> 1, lane = t & 31, warp = t >> 5;
-    const int c0 = blockIdx.x * 16 + u * 8;
-    constexpr int RSTEP = NT / 2;
-    // Launched early (programmatic dependent launch), this kernel may start while the kernel before
-    // it in the stream is still finishing: until that one is complete it only asks the L2 for its
-    // slice of A (a hint; no value is read), then it waits.  h and z^T are touched after the wait.
-    if (u == 0) {
-        for (int i = rl; i < d; i += RSTEP) prefetch_l2(A + (size_t)i * r + c0);
+    int rank = 0;
+#pragma unroll
+    for (int s = 0; s < 32; ++s) {
+        const uint32_t o = __shfl_sync(0xffffffffu, key, s);
+        rank += (o > key || (o == key && s < lane)) ? 1 : 0;
     }
+    const unsigned hit = __ballot_sync(0xffffffffu, rank == k - 1);
+    return __shfl_sync(0xffffffffu, key, __ffs(hit) - 1);
+}
+
+// The same for small k by k rounds of "take the maximum out": cheaper than counting up to about a dozen.
+__device__ __forceinline__ uint32_t warp_kth_largest_rounds(uint32_t key, int k, int lane)
+{
+    uint32_t kth = 0u;
+    for (int j = 0; j < k; ++j) {
+        kth = warp_max_u32(key);
+        const unsigned eq = __ballot_sync(0xffffffffu, key == kth);
+        if (lane == __ffs(eq) - 1) key = 0u;
+    }
+    return kth;
+}
+__device__ __forceinline__ uint32_t warp_kth_largest_any(uint32_t key, int k, int lane)
+{
+    return k <= 12 ? warp_kth_largest_rounds(key, k, lane) : warp_kth_largest(key, k, lane);
+}
+
+// The same over 64 values, two per lane (value a has index lane, value b index lane + 32).
+__device__ __forceinline__ uint32_t warp_kth_largest64(uint32_t a, uint32_t b, int k, int lane)
+{
+    int ra = 0, rb = 0;
+#pragma unroll
+    for (int s = 0; s < 32; ++s) {
+        const uint32_t oa = __shfl_sync(0xffffffffu, a, s);
+        const uint32_t ob = __shfl_sync(0xffffffffu, b, s);
+        ra += (oa > a || (oa == a && s < lane)) ? 1 : 0;
+        ra += (ob > a) ? 1 : 0;
+        rb += (oa >= b) ? 1 : 0;
+        rb += (ob > b || (ob == b && s < lane)) ? 1 : 0;
+    }
+    const unsigned hit_a = __ballot_sync(0xffffffffu, ra == k - 1);
+    const unsigned hit_b = __ballot_sync(0xffffffffu, rb == k - 1);
+    const uint32_t va = __shfl_sync(0xffffffffu, a, hit_a ? __ffs(hit_a) - 1 : 0);
+    const uint32_t vb = __shfl_sync(0xffffffffu, b, hit_b ? __ffs(hit_b) - 1 : 0);
+    return hit_a ? va : vb;
+}
+
+// n candidates in shared memory, in any order, distinct ids.  The warp writes the min(n, k)
+// best in order to (ok, oi) and pads up to k with empty entries.  By counting: a candidate's
+// place is the number of candidates ahead of it.
+__device__ __forceinline__ void warp_rank_select(const uint32_t* ck, const int* ci, int n, int k, uint32_t* ok,
+                                                 int* oi, int lane)
+{
+    for (int base = 0; base < n; base += 32) {
+        const int i = base + lane;
+        const uint32_t mk = i < n ? ck[i] : 0u;
+        const int mi = i < n ? ci[i] : kNoId;
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const uint32_t kj = ck[j];
+            const int ij = ci[j];
+            rank += (kj > mk || (kj == mk && ij < mi)) ? 1 : 0;
+        }
+        if (i < n && rank < k) { ok[rank] = mk; oi[rank] = mi; }
+    }
+    for (int j = n + lane; j < k; j += 32) { ok[j] = 0u; oi[j] = kNoId; }
+}
+
+// is (ka, ia) strictly after (kb, ib) in the order, i.e. a worse candidate?
+__device__ __forceinline__ bool after(uint32_t ka, int ia, uint32_t kb, int ib)
+{
+    return ka < kb || (ka == kb && ia > ib);
+}
+// is (ka, ia) a better candidate than (kb, ib)?
+__device__ __forceinline__ bool better(uint32_t ka, int ia, uint32_t kb, int ib)
+{
+    return ka > kb || (ka == kb && ia < ib);
+}
+
+// ------------------------------------------------------------------------------------------
+// The code z (or, for the full-rank head, h itself) reaches the head kernels in one of four forms:
+//   kCodeF32     fp32 [K][2]: entry (j, m) is z[m][j] (row 1 zero when M = 1): the FMA kernel
+//   kCodePacked  fragments, one part: rows 0-7 hold the value rounded to bf16 and rows 8-15 the
+//                rounding remainders of those same rows, so ONE instruction multiplies both
+//                (M <= 8; the two halves of its result are summed at the end)
+//   kCodeSplit   fragments, two parts: value and remainder of up to 16 rows (two instructions)
+//   kCodePlain   fragments, one part: up to 16 rows that are exact in bf16 (the full-rank head)
+// Fragments: word (kb, part, lane, reg) holds, for the 16-row block kb of the streamed matrix
+// (contraction indices 16 kb .. 16 kb + 15), the two bf16 values
+//     row  = (lane >> 2) + 8 (reg & 1),   index = 16 kb + 2 (lane & 3) + 8 (reg >> 1), + 1
+// (the lower index in the lower half): the "A" operand of mma.m16n8k16 as lane `lane` wants it.
+__host__ __device__ __forceinline__ size_t zfrag_word(int kb, int zparts, int part, int row, int idx16)
+{
+    const int lane = (row & 7) * 4 + ((idx16 & 7) >> 1);
+    const int reg = ((idx16 >> 3) << 1) | (row >> 3);
+    return (((size_t)kb * zparts + part) * 32 + lane) * 4 + reg;
+}
+
+// z = h A for up to 16 rows.  Grid (S, column tiles of 32), cluster (S, 1, 1): the CTAs of a
+// cluster split the d rows of A, each of their four warps takes a contiguous run of 16-row
+// blocks, and the partial tiles meet in the shared memory of the cluster's first CTA, which
+// rounds and writes the fragments.  Sums run in a fixed order: results do not depend on timing.
+struct CodeParams {
+    const bf16* h;
+    const bf16* A;
+    int M, d, r;
+    int S;            // K splits = CTAs per cluster
+    int nkb;          // 16-row blocks of A: ceil(d / 16)
+    int fmt;          // kCodeF32, kCodePacked or kCodeSplit
+    uint32_t* zfrag;  // the code in that form
+};
+
+static constexpr int kCodePitch = 80;            // bytes between two rows of the A slice in shared memory: 5 units (odd)
+static constexpr int kCodeChunkRows = 1024;      // rows of A a CTA holds at a time
+
+__global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
+{
+    __shared__ __align__(16) float wt[4][16 * 32];      // the warps' partial tiles
+    __shared__ __align__(16) float ct[8][16 * 32];      // the cluster's partial tiles (used in its first CTA)
+    extern __shared__ __align__(128) unsigned char aslice[];     // [rows][kCodePitch]: 32 columns of A
+    pdl_launch_dependents();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int rank = blockIdx.x;
+    const int j0 = blockIdx.y * 32;
+    const int d = p.d, r = p.r;
+    // this CTA's run of 16-row blocks, in chunks that fit the shared memory
+    const int cta_kb0 = (int)((long long)p.nkb * rank / p.S), cta_kb1 = (int)((long long)p.nkb * (rank + 1) / p.S);
+    auto fetch = [&](int kb0, int kb1) {
+        // weights may be read before the kernel ahead in the stream has finished: they are final before
+        // the call is made (the contract of the library); only h comes from that kernel
+        const int rows = 16 * (kb1 - kb0);
+        for (int idx = tid; idx < rows * 4; idx += 128) {
+            const int row = idx >> 2, u = idx & 3;
+            const int grow = min(16 * kb0 + row, d - 1);             // rows past d re-read the last row (their h is zero)
+            const int col = min(j0 + 8 * u, r - 8);                  // a ragged last tile re-reads the last columns
+            cp_async16(aslice + (size_t)row * kCodePitch + u * 16, p.A + (size_t)grow * r + col);
+        }
+        cp_async_commit();
+    };
+    const int chunk_kbs = kCodeChunkRows / 16;
+    fetch(cta_kb0, min(cta_kb1, cta_kb0 + chunk_kbs));
     pdl_wait();
 
-    float acc[MT][8];
+    float acc[4][4];
 #pragma unroll
-    for (int m = 0; m < MT; ++m)
+    for (int e = 0; e < 4; ++e)
 #pragma unroll
-        for (int c = 0; c < 8; ++c) acc[m][c] = 0.f;
+        for (int c = 0; c < 4; ++c) acc[e][c] = 0.f;
+    const uint32_t lane_off = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * kCodePitch + (uint32_t)(lane >> 4) * 16u;
+    const uint32_t as_s = smem_u32(aslice);
 
-    for (int i0 = rl; i0 < d; i0 += RSTEP * RB) {
-        uint4 a[RB];
-        float hv[MT][RB];
+    for (int c0 = cta_kb0; c0 < cta_kb1; c0 += chunk_kbs) {
+        const int c1 = min(cta_kb1, c0 + chunk_kbs);
+        if (c0 > cta_kb0) { __syncthreads(); fetch(c0, c1); }
+        // the warp's blocks of this chunk; their h fragments are the only loads that wait for the kernel ahead
+        const int n = c1 - c0;
+        const int wb0 = c0 + n * warp / 4, wb1 = c0 + n * (warp + 1) / 4;
+        cp_async_wait_pending(0);
+        __syncthreads();
+        for (int kb = wb0; kb < wb1; kb += 8) {
+            uint4 hf[8];
 #pragma unroll
-        for (int j = 0; j < RB; ++j) {
-            const int i = i0 + j * RSTEP;
-            a[j] = (i < d) ? __ldg(reinterpret_cast<const uint4*>(A + (size_t)i * r + c0)) : make_uint4(0u, 0u, 0u, 0u);
+            for (int i = 0; i < 8; ++i) {
+                const int k0 = 16 * (kb + i) + 2 * t;
+                const bool on = kb + i < wb1;
+                const bool lo_ok = on && k0 < d, hi_ok = on && k0 + 8 < d;
+                const uint32_t* h0 = reinterpret_cast<const uint32_t*>(p.h + (size_t)g * d + k0);
+                const uint32_t* h1 = reinterpret_cast<const uint32_t*>(p.h + (size_t)(g + 8) * d + k0);
+                hf[i].x = (g < p.M && lo_ok) ? __ldcg(h0) : 0u;
+                hf[i].y = (g + 8 < p.M && lo_ok) ? __ldcg(h1) : 0u;
+                hf[i].z = (g < p.M && hi_ok) ? __ldcg(h0 + 4) : 0u;
+                hf[i].w = (g + 8 < p.M && hi_ok) ? __ldcg(h1 + 4) : 0u;
+            }
 #pragma unroll
-            for (int m = 0; m < MT; ++m) hv[m][j] = (i < d && m < M) ? __bfloat162float(h[(size_t)m * d + i]) : 0.f;
-        }
-#pragma unroll
-        for (int j = 0; j < RB; ++j) {
-            const uint32_t w[4] = {a[j].x, a[j].y, a[j].z, a[j].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xffff0000u);
-#pragma unroll
-                for (int m = 0; m < MT; ++m) {
-                    acc[m][2 * e] = fmaf(hv[m][j], lo, acc[m][2 * e]);
-                    acc[m][2 * e + 1] = fmaf(hv[m][j], hi, acc[m][2 * e + 1]);
+            for (int i = 0; i < 8; ++i) {
+                if (kb + i < wb1) {
+                    const uint32_t a = as_s + (uint32_t)(kb + i - c0) * 16u * kCodePitch + lane_off;
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b0, b1, b2, b3, a);
+                    mma_bf16(acc[0], hf[i], b0, b1);
+                    mma_bf16(acc[1], hf[i], b2, b3);
+                    ldmatrix_x4_trans(b0, b1, b2, b3, a + 32u);
+                    mma_bf16(acc[2], hf[i], b0, b1);
+                    mma_bf16(acc[3], hf[i], b2, b3);
                 }
             }
         }
     }
-    // the 16 row lanes of a warp share a unit: fold them, then the warps through shared memory
+    // tile e of the instruction holds columns 8 e .. 8 e + 7 of the 32: lane (g, t) has columns
+    // 8 e + 2 t, + 1 for rows g (values 0, 1) and g + 8 (values 2, 3)
+    {
 #pragma unroll
-    for (int m = 0; m < MT; ++m)
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            float v = acc[m][c];
-            v += __shfl_xor_sync(0xffffffffu, v, 2);
-            v += __shfl_xor_sync(0xffffffffu, v, 4);
-            v += __shfl_xor_sync(0xffffffffu, v, 8);
-            v += __shfl_xor_sync(0xffffffffu, v, 16);
-            acc[m][c] = v;
+        for (int e = 0; e < 4; ++e) {
+            *reinterpret_cast<float2*>(&wt[warp][g * 32 + 8 * e + 2 * t]) = make_float2(acc[e][0], acc[e][1]);
+            *reinterpret_cast<float2*>(&wt[warp][(g + 8) * 32 + 8 * e + 2 * t]) = make_float2(acc[e][2], acc[e][3]);
         }
-    if (lane < 2) {
-#pragma unroll
-        for (int m = 0; m < MT; ++m)
-#pragma unroll
-            for (int c = 0; c < 8; ++c) red[warp][m][lane * 8 + c] = acc[m][c];
     }
     __syncthreads();
-    if (t < MT * 16) {
-        const int m = t >> 4, c = t & 15;
-        float v = 0.f;
+    float4 v = *reinterpret_cast<const float4*>(&wt[0][tid * 4]);
 #pragma unroll
-        for (int w = 0; w < NT / 32; ++w) v += red[w][m][c];
-        zT[(size_t)(blockIdx.x * 16 + c) * MT + m] = v;
+    for (int w = 1; w < 4; ++w) {
+        const float4 o = *reinterpret_cast<const float4*>(&wt[w][tid * 4]);
+        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+    }
+    if (p.S > 1) {
+        // every CTA of the cluster drops its tile into slot `rank` of the first CTA's shared memory
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(&ct[rank][tid * 4])), "r"(0));
+        asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z),
+                     "f"(v.w)
+                     : "memory");
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        if (rank != 0) return;
+        v = *reinterpret_cast<const float4*>(&ct[0][tid * 4]);
+        for (int s = 1; s < p.S; ++s) {
+            const float4 o = *reinterpret_cast<const float4*>(&ct[s][tid * 4]);
+            v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+        }
+    }
+    // four consecutive columns of one row
+    const int row = tid >> 3, j = j0 + (tid & 7) * 4;
+    if (j >= r) return;
+    const float z[4] = {v.x, v.y, v.z, v.w};
+    if (p.fmt == kCodeF32) {
+        float* zf = reinterpret_cast<float*>(p.zfrag);
+        if (row < 2) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) zf[(size_t)(j + e) * 2 + row] = z[e];
+        }
+        return;
+    }
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const bf16 hb = __float2bfloat16_rn(z[e]);
+        const bf16 lb = __float2bfloat16_rn(z[e] - __bfloat162float(hb));
+        hi[e] = (uint32_t)__bfloat16_as_ushort(hb);
+        lo[e] = (uint32_t)__bfloat16_as_ushort(lb);
+    }
+#pragma unroll
+    for (int pr = 0; pr < 2; ++pr) {
+        const int jj = j + 2 * pr;
+        const uint32_t hw = hi[2 * pr] | (hi[2 * pr + 1] << 16), lw = lo[2 * pr] | (lo[2 * pr + 1] << 16);
+        if (p.fmt == kCodePacked) {
+            if (row < 8) {
+                p.zfrag[zfrag_word(jj >> 4, 1, 0, row, jj & 15)] = hw;
+                p.zfrag[zfrag_word(jj >> 4, 1, 0, row + 8, jj & 15)] = lw;
+            }
+        } else {
+            p.zfrag[zfrag_word(jj >> 4, 2, 0, row, jj & 15)] = hw;
+            p.zfrag[zfrag_word(jj >> 4, 2, 1, row, jj & 15)] = lw;
+        }
     }
 }
 
-// z^T = widened h^T for the full-rank head (no down-projection).
-__global__ void k_stream_widen_t(const bf16* __restrict__ h, int M, int MT, int d, float* __restrict__ zT)
+// The full-rank head has no down-projection: its "code" is h itself, exact in bf16
+// (kCodeF32 or kCodePlain).
+__global__ void k_stream_widen(const bf16* __restrict__ h, int M, int d, int nkb, int fmt, uint32_t* __restrict__ zfrag)
 {
     pdl_launch_dependents();
-    pdl_wait();          // launched early: the kernel before it may still read z^T
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= d * MT) return;
-    const int i = e / MT, m = e % MT;
-    zT[e] = (m < M) ? __bfloat162float(h[(size_t)m * d + i]) : 0.f;
+    pdl_wait();          // launched early: the kernel before it may still read the code
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (fmt == kCodeF32) {
+        if (w >= 2 * d) return;
+        const int j = w >> 1, m = w & 1;
+        reinterpret_cast<float*>(zfrag)[w] = m < M ? __bfloat162float(h[(size_t)m * d + j]) : 0.f;
+        return;
+    }
+    if (w >= nkb * 128) return;
+    const int kb = w >> 7, lane = (w >> 2) & 31, reg = w & 3;
+    const int row = (lane >> 2) + 8 * (reg & 1);
+    const int idx = 16 * kb + 2 * (lane & 3) + 8 * (reg >> 1);
+    uint32_t word = 0u;
+    if (row < M && idx < d) word = *reinterpret_cast<const uint32_t*>(h + (size_t)row * d + idx);
+    zfrag[w] = word;
 }
 
 // ------------------------------------------------------------------------------------------
-// The streaming head.  One CTA per V slab; thread = (column unit of 8 columns, row group).
-// Every thread keeps U 128-bit loads of its column unit in flight (rows g, g+RG, g+2RG, ...),
-// multiplies each arriving row by the code held in shared memory (packed FP32 FMAs) and
-// refills.  The row groups' partial sums meet in shared memory; the warps of the slab then
-// keep the running max / sum-exp / top-k per row (or store the logits).  The last CTA to
-// finish merges the per-slab records.
-__device__ __forceinline__ uint4 ldg_stream(const void* p)
+// One task of the last CTA's merge, run by one warp: kind 0 = the row's log-sum-exp from the
+// records' (maximum, sum-exp) pairs, kind 1 = its k best entries.  A lane owns the records lane,
+// lane + 32, ... (NL of them at most) and keeps what it loads in registers: one round trip to the L2.
+template <int NL>
+__device__ __forceinline__ void merge_task(const HeadParams& p, int row, int kind, int lane, float* lse_s, uint32_t* ok, int* oi,
+                                           uint32_t* mk, int* mi, int* cnt)
 {
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p));
-    return r;
+    const int P = p.ncta, RW = p.rec_words, k = p.k;
+    const float* rows = p.part + (size_t)row * P * RW;
+    if (kind == 0) {
+        float2 ms[NL];
+#pragma unroll
+        for (int q = 0; q < NL; ++q) {
+            const int s = lane + 32 * q;
+            ms[q] = s < P ? __ldcg(reinterpret_cast<const float2*>(rows + (size_t)s * RW)) : make_float2(-FLT_MAX, 0.f);
+        }
+        float gm = -FLT_MAX;
+#pragma unroll
+        for (int q = 0; q < NL; ++q) gm = fmaxf(gm, ms[q].x);
+        gm = warp_max(gm);
+        float gs = 0.f;
+#pragma unroll
+        for (int q = 0; q < NL; ++q) gs += ms[q].y * __expf(ms[q].x - gm);
+        gs = warp_sum(gs);
+        if (lane == 0) lse_s[row] = gm + __logf(gs);
+        return;
+    }
+    // the first three entries of every record (words 2..7), then the bound: at least k entries
+    // reach the k-th largest of the lanes' best first entries
+    float2 e0[NL];
+    float4 e12[NL];
+#pragma unroll
+    for (int q = 0; q < NL; ++q) {
+        const int s = lane + 32 * q;
+        e0[q] = make_float2(0.f, __int_as_float(kNoId));
+        e12[q] = make_float4(0.f, __int_as_float(kNoId), 0.f, __int_as_float(kNoId));
+        if (s < P) {
+            e0[q] = __ldcg(reinterpret_cast<const float2*>(rows + (size_t)s * RW + 2));
+            if (k >= 2) e12[q] = __ldcg(reinterpret_cast<const float4*>(rows + (size_t)s * RW + 4));
+        }
+    }
+    uint32_t hk = 0u;
+#pragma unroll
+    for (int q = 0; q < NL; ++q) hk = max(hk, __float_as_uint(e0[q].x));
+    const uint32_t kth = warp_kth_largest_any(hk, min(k, 32), lane);
+    if (lane == 0) *cnt = 0;
+    __syncwarp();
+#pragma unroll
+    for (int q = 0; q < NL; ++q) {
+        const uint32_t k0 = __float_as_uint(e0[q].x);
+        if (k0 != 0u && k0 >= kth) {
+            int pos = atomicAdd(cnt, 1);
+            if (pos < kMergeCand) { mk[pos] = k0; mi[pos] = __float_as_int(e0[q].y); }
+            const uint32_t k1 = __float_as_uint(e12[q].x);
+            if (k >= 2 && k1 != 0u && k1 >= kth) {          // the record's list is in order: rarely more than one entry
+                pos = atomicAdd(cnt, 1);
+                if (pos < kMergeCand) { mk[pos] = k1; mi[pos] = __float_as_int(e12[q].y); }
+                const uint32_t k2 = __float_as_uint(e12[q].z);
+                if (k >= 3 && k2 != 0u && k2 >= kth) {
+                    pos = atomicAdd(cnt, 1);
+                    if (pos < kMergeCand) { mk[pos] = k2; mi[pos] = __float_as_int(e12[q].w); }
+                    const float* rec = rows + (size_t)(lane + 32 * q) * RW;
+                    for (int j = 3; j < k; ++j) {
+                        const float2 en = __ldcg(reinterpret_cast<const float2*>(rec + 2 + 2 * j));
+                        const uint32_t kj = __float_as_uint(en.x);
+                        if (kj == 0u || kj < kth) break;
+                        pos = atomicAdd(cnt, 1);
+                        if (pos < kMergeCand) { mk[pos] = kj; mi[pos] = __float_as_int(en.y); }
+                    }
+                }
+            }
+        }
+    }
+    __syncwarp();
+    const int n = *cnt;
+    if (n <= kMergeCand) {
+        warp_rank_select(mk, mi, n, k, ok, oi, lane);
+    } else {
+        // slow path: k rounds over every entry of the row's records, each round taking the best
+        // entry after the previous winner
+        uint32_t lk = 0xffffffffu;
+        int li = -1;
+        for (int j = 0; j < k; ++j) {
+            uint32_t bk = 0u;
+            int bi = kNoId;
+            for (int s = lane; s < P; s += 32) {
+                const float* rec = rows + (size_t)s * RW;
+                for (int e = 0; e < k; ++e) {
+                    const float2 en = __ldcg(reinterpret_cast<const float2*>(rec + 2 + 2 * e));
+                    const uint32_t ke = __float_as_uint(en.x);
+                    const int ie = __float_as_int(en.y);
+                    if (ke != 0u && after(ke, ie, lk, li) && better(ke, ie, bk, bi)) { bk = ke; bi = ie; }
+                }
+            }
+            const uint32_t wk = warp_max_u32(bk);
+            const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
+            lk = wk;
+            li = (int)wi;
+            if (lane == 0) { ok[j] = wk; oi[j] = wk != 0u ? (int)wi : kNoId; }
+            if (wk == 0u) { lk = 0u; li = kNoId; }
+        }
+    }
 }
 
-template <int MT, int U>
-__global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const HeadParams p)
+// ------------------------------------------------------------------------------------------
+// Epilogue of both head kernels.  The slab's logits lie in shared memory: logit (row, column c) is
+// the sum over g < ngroups of lg[g * gstride + row * lpitch + c] (the FMA kernel leaves one partial
+// sum per row group).  Thread i looks after columns i, i + blockDim, ...
+//   (1) maxima of groups of eight threads; (2) a warp per row: the k-th largest of these maxima
+//   bounds the slab's k-th largest logit from below; (3) sum of exp against the slab's maximum,
+//   logits that reach the bound are parked; (4) a warp per row orders the parked candidates by
+//   counting and writes the slab's record; then the arrival ticket, and the last CTA merges the
+//   records of every row the same way.
+// Nothing here depends on the order in which threads or CTAs arrive: results are reproducible.
+template <int MT>
+__device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char* smem, unsigned char* scratch, unsigned char* merge_area,
+                                              const float* lg, int ngroups, int gstride, int lpitch, int ncols, int col_base)
+{
+    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(smem);
+    float* gmax_s = reinterpret_cast<float*>(smem + 64);      // [16 rows][64]: maxima of thread groups
+    float* tau_s = gmax_s + 16 * 64;                          // [16] candidates must reach this
+    float* cmax_s = tau_s + 16;                               // [16] the slab's maximum
+    int* cnt_s = reinterpret_cast<int*>(cmax_s + 16);         // [16] candidates parked
+    float* wsum_s = reinterpret_cast<float*>(cnt_s + 16);     // [16 rows][16 warps] sums of exp
+    uint32_t* ck = reinterpret_cast<uint32_t*>(scratch);      // [MT][kCand]
+    int* ci = reinterpret_cast<int*>(ck + MT * kCand);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nt = blockDim.x, nw = nt >> 5;
+    const int cta = blockIdx.x, k = p.k;
+    const int mrows = min(p.M, MT);
+    auto logit = [&](int row, int c) {
+        float x = lg[row * lpitch + c];
+        for (int gi = 1; gi < ngroups; ++gi) x += lg[gi * gstride + row * lpitch + c];
+        return x + 0.f;             // -0 becomes +0: keys and float compares then agree
+    };
+
+    if (p.mode == 1) {
+        for (int row = 0; row < mrows; ++row)
+            for (int c = tid; c < ncols; c += nt) p.logits[(size_t)row * p.V + col_base + c] = logit(row, c);
+        return;
+    }
+    // ---- (1)
+    for (int row = 0; row < mrows; ++row) {
+        float m = -FLT_MAX;
+        for (int c = tid; c < ncols; c += nt) m = fmaxf(m, logit(row, c));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
+        if ((lane & 7) == 0) gmax_s[row * 64 + warp * 4 + (lane >> 3)] = m;
+    }
+    __syncthreads();
+    // ---- (2)  Up to 16 candidates wanted, the maxima of slot pairs do (32 values, half the
+    // shuffles); beyond that all 64 slots are ranked.
+    for (int row = warp; row < mrows; row += nw) {
+        const uint32_t ka = f2key(gmax_s[row * 64 + lane]), kb2 = f2key(gmax_s[row * 64 + 32 + lane]);
+        const uint32_t kth = (k <= 16) ? warp_kth_largest_any(max(ka, kb2), k, lane) : warp_kth_largest64(ka, kb2, min(k, 64), lane);
+        const uint32_t mx = warp_max_u32(max(ka, kb2));
+        if (lane == 0) { tau_s[row] = key2f(kth); cmax_s[row] = key2f(mx); cnt_s[row] = 0; }
+    }
+    __syncthreads();
+    // ---- (3)
+    for (int row = 0; row < mrows; ++row) {
+        const float tau = tau_s[row], cm = cmax_s[row];
+        float s = 0.f;
+        for (int c = tid; c < ncols; c += nt) {
+            const float x = logit(row, c);
+            s += __expf(x - cm);
+            if (x >= tau) {
+                const int pos = atomicAdd(&cnt_s[row], 1);
+                if (pos < kCand) { ck[row * kCand + pos] = f2key(x); ci[row * kCand + pos] = col_base + c; }
+            }
+        }
+        s = warp_sum(s);
+        if (lane == 0) wsum_s[row * 16 + warp] = s;
+    }
+    __syncthreads();
+    // ---- (4)
+    const int P = p.ncta;
+    const int RW = p.rec_words;
+    for (int row = warp; row < mrows; row += nw) {
+        float* rec = p.part + ((size_t)row * P + cta) * RW;
+        {
+            const float s = warp_sum(lane < nw ? wsum_s[row * 16 + lane] : 0.f);      // fixed order: reproducible
+            if (lane == 0) *reinterpret_cast<float2*>(rec) = make_float2(cmax_s[row], s);
+        }
+        const int n = cnt_s[row];
+        if (n <= kCand) {
+            // the (key, id) pairs go straight into the record: rank j to words 2 + 2 j, 3 + 2 j
+            const uint32_t* rk = ck + row * kCand;
+            const int* ri = ci + row * kCand;
+            for (int base = 0; base < n; base += 32) {
+                const int i = base + lane;
+                const uint32_t mk = i < n ? rk[i] : 0u;
+                const int mi = i < n ? ri[i] : kNoId;
+                int rank = 0;
+                for (int j = 0; j < n; ++j) rank += better(rk[j], ri[j], mk, mi) ? 1 : 0;
+                if (i < n && rank < k) *reinterpret_cast<float2*>(rec + 2 + 2 * rank) = make_float2(__uint_as_float(mk), __int_as_float(mi));
+            }
+            for (int j = n + lane; j < k; j += 32) *reinterpret_cast<float2*>(rec + 2 + 2 * j) = make_float2(__uint_as_float(0u), __int_as_float(kNoId));
+        } else {
+            // Slow path (masses of equal logits, or logits in long ordered runs): k rounds over the
+            // row, each taking the best logit that comes after the previous winner in the order;
+            // nothing is kept between rounds but that winner.
+            uint32_t lk = 0xffffffffu;
+            int li = -1;
+            for (int j = 0; j < k; ++j) {
+                uint32_t bk = 0u;
+                int bi = kNoId;
+                for (int c = lane; c < ncols; c += 32) {
+                    const uint32_t ke = f2key(logit(row, c));
+                    const int ie = col_base + c;
+                    if (after(ke, ie, lk, li) && better(ke, ie, bk, bi)) { bk = ke; bi = ie; }
+                }
+                const uint32_t wk = warp_max_u32(bk);
+                const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
+                lk = wk;
+                li = (int)wi;
+                if (lane == 0) *reinterpret_cast<float2*>(rec + 2 + 2 * j) = make_float2(__uint_as_float(wk), __int_as_float(wk != 0u ? (int)wi : kNoId));
+                if (wk == 0u) { lk = 0u; li = kNoId; }      // nothing left: later rounds stay empty
+            }
+        }
+    }
+
+    // ---- arrival: the last CTA merges the records of every row
+    __syncthreads();
+    if (tid == 0) *s_ticket = ticket_take(p.ticket);
+    __syncthreads();
+    if (*s_ticket != (unsigned)(p.ncta - 1)) return;
+
+    // Two tasks per row, a warp each: the row's log-sum-exp, and its k best entries.
+    float* lse_s = reinterpret_cast<float*>(merge_area);                 // [16]
+    uint32_t* ok_all = reinterpret_cast<uint32_t*>(lse_s + 16);          // [16 rows][32] ordered keys
+    int* oi_all = reinterpret_cast<int*>(ok_all + 16 * 32);              // [16 rows][32] their ids
+    uint32_t* mk = reinterpret_cast<uint32_t*>(oi_all + 16 * 32) + warp * 2 * kMergeCand;     // this warp's candidates
+    int* mi = reinterpret_cast<int*>(mk + kMergeCand);
+    for (int task = warp; task < 2 * p.M; task += nw) {
+        const int row = task >> 1;
+        if (P <= 5 * 32) merge_task<5>(p, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+        else merge_task<kMergeLists>(p, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+    }
+    __syncthreads();
+    for (int e = tid; e < p.M * k; e += nt) {
+        const int row = e / k, j = e - row * k;
+        p.ids[e] = oi_all[row * 32 + j];
+        p.logprobs[e] = key2f(ok_all[row * 32 + j]) - lse_s[row];
+    }
+    if (tid == 0) *p.ticket = 0;
+}
+
+// Common prologue of the head kernels: let the next kernel come up, ask the L2 for the first rows
+// of the slab, then wait for the kernel that writes the code.
+__device__ __forceinline__ void head_prologue(const HeadParams& p, const char* slab, int my_units, size_t Vb)
+{
+    pdl_launch_dependents();
+    if (p.wait_prev) {
+        // Until the code is there this CTA can only wait, and while it waits HBM would idle: ask the
+        // L2 for the first rows of the slab (a hint: no value is read before the wait, so whatever
+        // precedes this call in the stream may still be writing its results).
+        if (p.pf_rows > 0 && my_units > 0) {
+            const int seg_bytes = my_units * 16;
+            const int lines = (seg_bytes + 127) / 128 + 1;          // the row segment need not start on a line
+            for (int i = threadIdx.x; i < p.pf_rows * lines; i += blockDim.x) {
+                const int r = i / lines, l = i - r * lines;
+                prefetch_l2(slab + (size_t)r * Vb + min(l * 128, seg_bytes - 1));
+            }
+        }
+        pdl_wait();
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// One or two rows.  One CTA per V slab; thread = (column unit of 8 columns, row group).  Every
+// thread keeps 16 loads of its unit in flight (rows g, g + RG, g + 2 RG, ...) in two alternating
+// register sets, so that a wait for the older set never waits for loads issued after it,
+// multiplies each arriving row by the code held in shared memory as (z, z) pairs (packed FP32
+// FMAs) and refills.  The row groups' partial sums meet in shared memory.
+template <int MT>
+__global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(smem);
-    uint32_t* sel_s = reinterpret_cast<uint32_t*>(smem + 128);           // [16 warps][32 keys, 32 ids]
-    float* ep_s = reinterpret_cast<float*>(smem + 128 + 16 * 64 * 4);    // [MT][kMaxColWarps][66]
-    float* red = ep_s + MT * kMaxColWarps * 66;                          // [RG][MT][ct*8]
+    unsigned char* zarea = smem + ((kEpFixedBytes + 127) / 128) * 128;
+    float2* zs = reinterpret_cast<float2*>(zarea);              // [K][MT] (z, z) pairs
+    float* red = reinterpret_cast<float*>(zarea + p.zarea_bytes);   // [RG][MT][lpitch] partial sums, then the epilogue's lists
+    const int tid = threadIdx.x;
     const int CT = p.ct, RG = p.rg;
-    const int pass_cols = CT * 8;
-    float2* zs = reinterpret_cast<float2*>(red + (size_t)RG * MT * pass_cols);   // [kc][MT] (z, z) pairs
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    uint32_t* sel_k = sel_s + warp * 64;             // this warp's selection output
-    int* sel_i = reinterpret_cast<int*>(sel_k + 32);
-    const int g = tid / CT, c = tid - g * CT;        // row group, column unit inside the pass
-    const int NW = CT >> 5;                          // warps across a pass
-    const int cw = warp - g * NW;                    // this warp's position across the pass
+    const int g = tid / CT, c = tid - g * CT;                   // row group, column unit
     const int cta = blockIdx.x;
-    const int K = p.K, V = p.V, k = p.k;
-    const int stepU = RG * U;
-
-    // ---- this CTA's slab and its passes
+    const int K = p.K;
+    const size_t Vb = (size_t)p.V * sizeof(bf16);
     const int my_units = p.units_base + (cta < p.units_rem ? 1 : 0);
     const int unit0 = cta * p.units_base + min(cta, p.units_rem);
-    const int npass = (my_units + p.pass_units - 1) / p.pass_units;
-    const int units_per_pass = npass ? (my_units + npass - 1) / npass : 0;
+    const char* slab = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
+    const int lpitch = CT * 8;
 
-    // Two sets of UH loads each: one set is consumed while the other is in flight, so a wait
-    // for the older set never waits for loads issued after it.
-    constexpr int UH = U / 2;
+    constexpr int U = kFmaLoads, UH = U / 2;
+    const bool active = g < RG && c < my_units;
+    const char* base = slab + (size_t)c * 16;
+    const int stepU = RG * U;
+    const uint64_t pol = policy_evict_first();
+    // The first rows of the weights go out before the kernel ahead in the stream is waited for: they
+    // are final before the call is made (the contract of the library); only the code depends on that
+    // kernel.  The rows behind them are asked into the L2 meanwhile.
     uint4 q[2][UH];
-    auto prologue = [&](int pass) {
-        const int pu0 = pass * units_per_pass;
-        const int pun = min(units_per_pass, my_units - pu0);
-        const bf16* base = p.B + (size_t)(unit0 + pu0 + c) * 8;
+    if (active) {
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh)
 #pragma unroll
             for (int j = 0; j < UH; ++j) {
                 const int row = g + (hh * UH + j) * RG;
-                q[hh][j] = (c < pun && row < K) ? ldg_stream(base + (size_t)row * V) : make_uint4(0u, 0u, 0u, 0u);
+                q[hh][j] = row < K ? ldg_stream(base + (size_t)row * Vb, pol) : make_uint4(0u, 0u, 0u, 0u);
             }
-    };
-    if (npass > 0) prologue(0);
-    // the weights are on their way; let the next kernel in the stream come up behind this one,
-    // then wait for the kernel that writes the code
-    pdl_launch_dependents();
-    if (p.wait_prev) {
-        // Until the code is there this CTA can only wait, and while it waits HBM idles: ask the L2
-        // for the rows of the slab that come next (a hint; the loads of the main loop then hit the
-        // L2).  Launched early behind a kernel that still runs, the wait is several microseconds.
-        if (p.pf_rows > 0 && npass > 0) {
-            const int pun0 = min(units_per_pass, my_units);
-            const int lines = (pun0 * 16 + 127) / 128 + 1;          // the slab's row segment need not start on a line
-            const int r0 = min(K, stepU), r1 = min(K, stepU + p.pf_rows);
-            const char* seg = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
-            const size_t row_bytes = (size_t)V * sizeof(bf16);
-            const int last = pun0 * 16 - 1;                          // last byte of the row segment
-            for (int i = tid; i < (r1 - r0) * lines; i += blockDim.x) {
-                const int r = r0 + i / lines, l = i - (i / lines) * lines;
-                prefetch_l2(seg + (size_t)r * row_bytes + min(l * 128, last));
-            }
+    }
+    head_prologue(p, slab + (size_t)min(K, stepU) * Vb, my_units, Vb);
+    for (int i = tid; i < 16 * 64; i += blockDim.x) reinterpret_cast<float*>(smem + 64)[i] = -FLT_MAX;
+    // the code first (the main loop cannot start without it): fp32 [K][2] in global memory -> (z, z) pairs
+    {
+        const float* zf = reinterpret_cast<const float*>(p.zfrag);
+        for (int e = tid; e < K * MT; e += blockDim.x) {
+            const int j = e / MT, m = e - j * MT;
+            const float zv = __ldcg(zf + (size_t)j * 2 + m);
+            zs[e] = make_float2(zv, zv);
         }
-        pdl_wait();
     }
+    __syncthreads();
 
-    float run_max[MT], run_sum[MT];
-    uint32_t lst_k[MT];                              // lane j < k: key of the j-th best so far
-    int lst_i[MT];
-    bool mine[MT];                                   // rows whose softmax / top-k this warp keeps
+    float2 acc[MT][4];
 #pragma unroll
-    for (int m = 0; m < MT; ++m) {
-        run_max[m] = -FLT_MAX; run_sum[m] = 0.f; lst_k[m] = 0; lst_i[m] = kNoId;
-        mine[m] = (m % RG) == g;
-    }
-
-    for (int pass = 0; pass < npass; ++pass) {
-        const int pu0 = pass * units_per_pass;
-        const int pun = min(units_per_pass, my_units - pu0);
-        const bool active = c < pun;
-        const bf16* base = p.B + (size_t)(unit0 + pu0 + c) * 8;
-        float2 acc[MT][4];
+    for (int m = 0; m < MT; ++m)
 #pragma unroll
-        for (int m = 0; m < MT; ++m)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[m][e] = make_float2(0.f, 0.f);
-
-        // rows row, row + RG, ... (U of them): multiply what has arrived, then refill
-        auto block = [&](int row, int kc0, int kend, auto checked) {
-            constexpr bool kChecked = decltype(checked)::value;
+        for (int e = 0; e < 4; ++e) acc[m][e] = make_float2(0.f, 0.f);
+    if (active) {
+        for (int row = g; row < K; row += stepU) {
+            const bool checked = row - g + 2 * stepU > K;       // this block or its refills reach past K
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll
                 for (int j = 0; j < UH; ++j) {
                     const int rj = row + (hh * UH + j) * RG;
-                    if (!kChecked || rj < kend) {
+                    if (!checked || rj < K) {
                         const uint32_t w[4] = {q[hh][j].x, q[hh][j].y, q[hh][j].z, q[hh][j].w};
                         float2 b2[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
                             b2[e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
-                        const float2* zr = zs + (size_t)(rj - kc0) * MT;
+                        const float2* zr = zs + (size_t)rj * MT;
 #pragma unroll
                         for (int m = 0; m < MT; ++m) {
                             const float2 z2 = zr[m];
@@ -356,361 +784,376 @@ __global__ void __launch_bounds__(MT <= 4 ? 512 : 256, 1) k_stream_head(const He
 #pragma unroll
                 for (int j = 0; j < UH; ++j) {
                     const int nr = row + (hh * UH + j) * RG + stepU;
-                    if (!kChecked || nr < K) q[hh][j] = ldg_stream(base + (size_t)nr * V);
-                }
-            }
-        };
-
-        for (int kc0 = 0; kc0 < K; kc0 += p.kc) {
-            const int kend = min(K, kc0 + p.kc);
-            if (pass == 0 || p.kc < K) {
-                // bring this chunk of the code into shared memory as (z, z) pairs
-                if (kc0 > 0 || pass > 0) __syncthreads();
-                const float* src = p.zT + (size_t)kc0 * MT;
-                for (int e = tid; e < (kend - kc0) * MT; e += blockDim.x) {
-                    const float zv = __ldcg(src + e);
-                    zs[e] = make_float2(zv, zv);
-                }
-                __syncthreads();
-            }
-            if (active) {
-                for (int row = kc0 + g; row < kend; row += stepU) {
-                    // unchecked while this block and the next one lie wholly inside K
-                    if (row - g + 2 * stepU <= K) block(row, kc0, kend, std::false_type());
-                    else block(row, kc0, kend, std::true_type());
+                    if (!checked || nr < K) q[hh][j] = ldg_stream(base + (size_t)nr * Vb, pol);
                 }
             }
         }
-        // ---- the row groups' partial sums meet in shared memory
-        if (active) {
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                float* dst = red + ((size_t)g * MT + m) * pass_cols + c * 8;
-                *reinterpret_cast<float4*>(dst) = make_float4(acc[m][0].x, acc[m][0].y, acc[m][1].x, acc[m][1].y);
-                *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[m][2].x, acc[m][2].y, acc[m][3].x, acc[m][3].y);
-            }
-        }
-        // next pass's first loads fly while this pass's logits are reduced
-        if (pass + 1 < npass) prologue(pass + 1);
-        __syncthreads();
-
-        const int col = (unit0 + pu0 + c) * 8;       // first vocabulary id of this thread
+    }
+    if (g < RG && c < CT) {
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
-            if (!mine[m] || m >= p.M) continue;
-            float l[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) l[e] = 0.f;
-            if (active) {
-                for (int gg = 0; gg < RG; ++gg) {
-                    const float* src = red + ((size_t)gg * MT + m) * pass_cols + c * 8;
-                    const float4 a = *reinterpret_cast<const float4*>(src);
-                    const float4 b = *reinterpret_cast<const float4*>(src + 4);
-                    l[0] += a.x; l[1] += a.y; l[2] += a.z; l[3] += a.w;
-                    l[4] += b.x; l[5] += b.y; l[6] += b.z; l[7] += b.w;
-                }
-            }
-            if (p.mode == 1) {
-                if (active) {
-                    float* dst = p.logits + (size_t)m * V + col;
-                    *reinterpret_cast<float4*>(dst) = make_float4(l[0], l[1], l[2], l[3]);
-                    *reinterpret_cast<float4*>(dst + 4) = make_float4(l[4], l[5], l[6], l[7]);
-                }
-                continue;
-            }
-            // online softmax + running top-k of this warp's columns
-            float tmax = -FLT_MAX;
-            if (active) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) tmax = fmaxf(tmax, l[e]);
-            }
-            const float wmax = warp_max(tmax);
-            const float nm = fmaxf(run_max[m], wmax);
-            float ts = 0.f;
-            if (active) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) ts += __expf(l[e] - nm);
-            }
-            run_sum[m] = run_sum[m] * __expf(run_max[m] - nm) + warp_sum(ts);
-            run_max[m] = nm;
-            // skip the selection when nothing here beats the current k-th best
-            const uint32_t kth = __shfl_sync(0xffffffffu, lst_k[m], k - 1);
-            if (f2key(wmax) < kth) continue;
-            // this lane's list: its eight new logits in order, then its entry of the running list
-            uint32_t ck[9];
-            int ci[9];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) { ck[e] = active ? f2key(l[e]) : 0u; ci[e] = active ? col + e : kNoId; }
-            sort8(ck, ci);
-            ck[8] = lst_k[m];
-            ci[8] = lst_i[m];
-#pragma unroll
-            for (int e = 7; e >= 0; --e) order2(ck[e], ci[e], ck[e + 1], ci[e + 1]);
-            sel_k[lane] = 0u;
-            sel_i[lane] = kNoId;
-            __syncwarp();
-            warp_topk_regs<9>(ck, ci, k, sel_k, sel_i);
-            __syncwarp();
-            lst_k[m] = sel_k[lane];
-            lst_i[m] = sel_i[lane];
-            __syncwarp();
+            float* dst = red + ((size_t)g * MT + m) * lpitch + c * 8;
+            *reinterpret_cast<float4*>(dst) = make_float4(acc[m][0].x, acc[m][0].y, acc[m][1].x, acc[m][1].y);
+            *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[m][2].x, acc[m][2].y, acc[m][3].x, acc[m][3].y);
         }
-        if (pass + 1 < npass) __syncthreads();       // the partial sums may be overwritten now
-    }
-    if (p.mode == 1) return;
-
-    // ---- fold the warps across the slab into one record per (row, slab)
-    // ep_s: per (row, warp) 66 words: max, sum-exp, 32 keys, 32 ids
-#pragma unroll
-    for (int m = 0; m < MT; ++m) {
-        if (!mine[m] || m >= p.M) continue;
-        float* rec = ep_s + ((size_t)m * kMaxColWarps + cw) * 66;
-        if (lane == 0) { rec[0] = run_max[m]; rec[1] = run_sum[m]; }
-        rec[2 + lane] = __uint_as_float(lst_k[m]);
-        rec[34 + lane] = __int_as_float(lst_i[m]);
     }
     __syncthreads();
-    const int P = p.ncta;
-    const int RW = p.rec_words;
-    if (cw == 0) {
-        // the lanes share out the NW sorted lists: 32 / NW lanes per list, a run of each list per lane
-        const int lpl = 32 / NW;
-        const int seg = (k + lpl - 1) / lpl;
-        const int lw = lane / lpl, ls = lane - lw * lpl;
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            if (!mine[m] || m >= p.M) continue;
-            const float* rows = ep_s + (size_t)m * kMaxColWarps * 66;
-            float cm = -FLT_MAX, cs = 0.f;
-            if (MT > 1 || NW > 4) {
-                // lane w takes warp w's (max, sum-exp); measured better than the loop except for one row
-                // with up to four warps
-                const float wm = lane < NW ? rows[lane * 66] : -FLT_MAX;
-                cm = warp_max(wm);
-                cs = warp_sum(lane < NW ? rows[lane * 66 + 1] * __expf(wm - cm) : 0.f);
-            } else {
-                for (int w = 0; w < NW; ++w) cm = fmaxf(cm, rows[w * 66]);
-                for (int w = 0; w < NW; ++w) cs += rows[w * 66 + 1] * __expf(rows[w * 66] - cm);
-            }
-            const int first = ls * seg;
-            const int len = (lw < NW && first < k) ? min(seg, k - first) : 0;
-            const int lwc = lw < NW ? lw : 0;
-            const uint32_t* lk = reinterpret_cast<const uint32_t*>(rows + lwc * 66 + 2 + first);
-            const int* li = reinterpret_cast<const int*>(rows + lwc * 66 + 34 + first);
-            sel_k[lane] = 0u;
-            sel_i[lane] = kNoId;
-            __syncwarp();
-            warp_topk_smem(lk, li, len, k, sel_k, sel_i);
-            __syncwarp();
-            const uint32_t ok = sel_k[lane];
-            const int oi = sel_i[lane];
-            __syncwarp();
-            float* gp = p.part + ((size_t)m * P + cta) * RW;
-            if (lane == 0) { gp[0] = cm; gp[1] = cs; }
-            if (lane < k) {
-                gp[2 + lane] = __uint_as_float(ok);
-                gp[2 + k + lane] = __int_as_float(oi);
-            }
-        }
-        __threadfence();
-    }
-    __syncthreads();
-    if (tid == 0) *s_ticket = atomicAdd(p.ticket, 1u);
-    __syncthreads();
-    if (*s_ticket != (unsigned)(P - 1)) return;
-
-    // ---- last CTA: merge the P slab records of every row, a few rows per round
-    __threadfence();
-    float* mrg = red;                                // the reduction and code areas are idle now
-    __shared__ float lse_s[32];                      // a row's log-sum-exp, by the row's place in the round
-    uint32_t* stage_k = reinterpret_cast<uint32_t*>(ep_s);            // [rows][groups][32] keys, then ids
-    const int row_words = P * RW;
-    const int ngroups = (P + 31) >> 5;               // groups of 32 slabs, one warp each
-    const int nwarps = blockDim.x >> 5;
-    for (int m0 = 0; m0 < p.M; m0 += p.merge_rows) {
-        const int nrows = min(p.merge_rows, p.M - m0);
-        const int n4 = nrows * row_words / 4;
-        const float4* src = reinterpret_cast<const float4*>(p.part + (size_t)m0 * row_words);
-        float4* dst = reinterpret_cast<float4*>(mrg);
-        // batches of independent loads: the records sit in L2, one round trip per batch
-        for (int i0 = tid; i0 < n4; i0 += blockDim.x * 8) {
-            float4 t[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int i = i0 + j * blockDim.x;
-                t[j] = (i < n4) ? __ldcg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int i = i0 + j * blockDim.x;
-                if (i < n4) dst[i] = t[j];
-            }
-        }
-        __syncthreads();
-        // first level: a warp takes 32 slabs of one row, a lane per slab list
-        int* stage_i = reinterpret_cast<int*>(stage_k + (size_t)nrows * ngroups * 32);
-        for (int job = warp; job < nrows * ngroups; job += nwarps) {
-            const int rrow = job / ngroups, grp = job - rrow * ngroups;
-            const int s = grp * 32 + lane;
-            const float* rec = mrg + (size_t)rrow * row_words + (size_t)(s < P ? s : 0) * RW;
-            stage_k[(size_t)job * 32 + lane] = 0u;
-            stage_i[(size_t)job * 32 + lane] = kNoId;
-            __syncwarp();
-            warp_topk_smem(reinterpret_cast<const uint32_t*>(rec + 2), reinterpret_cast<const int*>(rec + 2 + k),
-                           s < P ? k : 0, k, stage_k + (size_t)job * 32, stage_i + (size_t)job * 32);
-        }
-        // meanwhile the warps at the other end take the rows' log-sum-exp (it needs no list)
-        if (warp >= nwarps - nrows) {
-            const int rrow = nwarps - 1 - warp;
-            const float* rows = mrg + (size_t)rrow * row_words;
-            float gm = -FLT_MAX;
-            for (int s = lane; s < P; s += 32) gm = fmaxf(gm, rows[(size_t)s * RW]);
-            gm = warp_max(gm);
-            float gs = 0.f;
-            for (int s = lane; s < P; s += 32) gs += rows[(size_t)s * RW + 1] * __expf(rows[(size_t)s * RW] - gm);
-            gs = warp_sum(gs);
-            if (lane == 0) lse_s[rrow] = gm + __logf(gs);
-        }
-        __syncthreads();
-        // second level: a warp per row folds the groups' lists and finishes the log-softmax
-        if (warp < nrows) {
-            const int m = m0 + warp;
-            const float lse = lse_s[warp];
-            const int lpl = 32 / ngroups;
-            const int seg = (k + lpl - 1) / lpl;
-            const int lw = lane / lpl, ls = lane - lw * lpl;
-            const int first = ls * seg;
-            const int len = (lw < ngroups && first < k) ? min(seg, k - first) : 0;
-            const size_t off = ((size_t)warp * ngroups + (lw < ngroups ? lw : 0)) * 32 + first;
-            sel_k[lane] = 0u;
-            sel_i[lane] = kNoId;
-            __syncwarp();
-            warp_topk_smem(stage_k + off, stage_i + off, len, k, sel_k, sel_i);
-            __syncwarp();
-            const uint32_t ok = sel_k[lane];
-            const int oi = sel_i[lane];
-            if (lane < k) {
-                p.ids[(size_t)m * k + lane] = oi;
-                p.logprobs[(size_t)m * k + lane] = key2f(ok) - lse;
-            }
-        }
-        __syncthreads();
-    }
-    if (tid == 0) *p.ticket = 0;
+    unsigned char* lists = reinterpret_cast<unsigned char*>(red + (size_t)RG * MT * lpitch);
+    slab_epilogue<MT>(p, smem, lists, zarea, red, RG, MT * lpitch, lpitch, my_units * 8, unit0 * 8);
 }
 
 // ------------------------------------------------------------------------------------------
-static int pick_mt(int M) { return M <= 1 ? 1 : M <= 2 ? 2 : M <= 4 ? 4 : 8; }
+// Three to sixteen rows.  One CTA per V slab, 14 warps.  The slab's rows arrive through a ring
+// of shared-memory stages (16 rows of the matrix each), filled by cp.async.  A warp owns 64 columns
+// of the slab (two such chunks when the slab is wider than 14 x 64 columns) and all K rows: per
+// stage it reads the "B" fragments of eight m16n8k16 instructions per chunk with ldmatrix.trans
+// (the row pitch is an odd number of 16-byte units, so the eight rows of a matrix fall into
+// distinct banks) and the code fragment from its own area of shared memory.  Lane (g, t) ends up
+// with the logits of rows g and g + 8 at columns 8 e + 2 t, 8 e + 2 t + 1 of every 8-column unit e
+// of its chunks.  MT = 8: rows 8-15 of the code fragment are the remainders of rows 0-7 (or zero),
+// and the two halves of the result are summed.
+template <int MT, int ZP, int NCH>
+__global__ void __launch_bounds__(512, 1) k_stream_head_mma(const HeadParams p)      // 512: at most 128 registers, so that a small CTA fits beside it
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* zarea = smem + ((kEpFixedBytes + 127) / 128) * 128;
+    unsigned char* ring = zarea + p.zarea_bytes;
 
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int nw = blockDim.x >> 5;
+    const int cta = blockIdx.x;
+    const int K = p.K;
+    const size_t Vb = (size_t)p.V * sizeof(bf16);
+
+    const int my_units = p.units_base + (cta < p.units_rem ? 1 : 0);
+    const int unit0 = cta * p.units_base + min(cta, p.units_rem);
+    const char* slab = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
+
+    head_prologue(p, slab, my_units, Vb);
+    for (int i = tid; i < 16 * 64; i += blockDim.x) reinterpret_cast<float*>(smem + 64)[i] = -FLT_MAX;
+
+    // ---- this thread's share of a stage: 16-byte pieces (row, unit), the same for every stage
+    constexpr int kMaxCopies = 8;
+    uint32_t src_off[kMaxCopies], dst_off[kMaxCopies];
+    const int pitch = p.pitch_units;                    // units between two rows of a stage (odd)
+    const uint32_t stage_bytes = 16u * (uint32_t)pitch * 16u;
+#pragma unroll
+    for (int i = 0; i < kMaxCopies; ++i) {
+        const int idx = tid + i * (int)blockDim.x;
+        const int row = my_units > 0 ? idx / my_units : 16;
+        const int c = idx - row * my_units;
+        src_off[i] = row < 16 ? (uint32_t)((size_t)row * Vb) + (uint32_t)c * 16u : 0xffffffffu;
+        dst_off[i] = ((uint32_t)row * (uint32_t)pitch + (uint32_t)c) * 16u;
+    }
+    const int nkb = p.nkb, NS = p.ns;
+    auto issue_stage = [&](int kb, int slot) {
+        if (kb < nkb) {
+            unsigned char* dst = ring + (size_t)slot * stage_bytes;
+            if (16 * kb + 16 <= K) {
+                const char* src = slab + (size_t)(16 * kb) * Vb;
+#pragma unroll
+                for (int i = 0; i < kMaxCopies; ++i)
+                    if (src_off[i] != 0xffffffffu) cp_async16(dst + dst_off[i], src + src_off[i]);
+            } else {
+                // the last block of a K that is no multiple of 16: rows past the end re-read the last
+                // row (their code entries are zero)
+                for (int idx = tid; idx < 16 * my_units; idx += blockDim.x) {
+                    const int row = idx / my_units, c = idx - row * my_units;
+                    cp_async16(dst + ((size_t)row * pitch + c) * 16, slab + (size_t)min(16 * kb + row, K - 1) * Vb + (size_t)c * 16);
+                }
+            }
+        }
+    };
+    // code fragments: whole in shared memory, or chunk by chunk through two buffers
+    const size_t kb_bytes = (size_t)ZP * 512;
+    const size_t zchunk_bytes = (size_t)p.kb_chunk * kb_bytes;
+    auto copy_zchunk = [&](int c) {
+        const int kb0 = c * p.kb_chunk;
+        if (kb0 >= nkb) return;
+        unsigned char* dst = zarea + (p.nchunks > 1 ? (size_t)(c & 1) * zchunk_bytes : 0);
+        const int n16 = (int)((size_t)(min(nkb, kb0 + p.kb_chunk) - kb0) * kb_bytes / 16);
+        const uint4* src = reinterpret_cast<const uint4*>(p.zfrag) + (size_t)kb0 * kb_bytes / 16;
+        for (int i = tid; i < n16; i += blockDim.x) cp_async16(dst + (size_t)i * 16, src + i);
+    };
+
+    // ---- the warp's chunks of 64 columns and its ldmatrix lane address inside a stage
+    bool chunk_on[NCH];
+    int cb[NCH];                                        // first unit of the chunk
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch) { cb[ch] = 8 * (warp + nw * ch); chunk_on[ch] = cb[ch] < my_units; }
+    // lane l gives the address of row (l & 7) of matrix (l >> 3): matrices 0, 1 are rows 0-7 and
+    // 8-15 of a unit, matrices 2, 3 the same rows of the next unit
+    const uint32_t lane_off = ((uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * (uint32_t)pitch + (uint32_t)(lane >> 4)) * 16u;
+    const uint32_t ring_s = smem_u32(ring);
+
+    float acc[NCH][8][4];
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[ch][e][c] = 0.f;
+
+    // ---- the pipeline: NS - 1 stages in flight
+    copy_zchunk(0);
+    for (int s = 0; s < NS - 1; ++s) { issue_stage(s, s); cp_async_commit(); }
+    int slot = 0, fill_slot = NS - 1;
+    int zc = 0, zkb0 = 0, zkb1 = min(nkb, p.kb_chunk);      // current chunk of the code
+    for (int kb = 0; kb < nkb; ++kb) {
+        cp_async_wait_pending(NS - 2);
+        __syncthreads();            // stage kb has landed for everyone; everyone is done with stage kb - 1
+        if (kb == zkb1) { ++zc; zkb0 = zkb1; zkb1 = min(nkb, zkb0 + p.kb_chunk); }
+        if (kb == zkb0 && p.nchunks > 1) copy_zchunk(zc + 1);
+        issue_stage(kb + NS - 1, fill_slot);
+        cp_async_commit();
+        if (++fill_slot == NS) fill_slot = 0;
+
+        const unsigned char* zbuf = zarea + (p.nchunks > 1 ? (size_t)(zc & 1) * zchunk_bytes : 0);
+        const uint4* zp = reinterpret_cast<const uint4*>(zbuf) + (size_t)(kb - zkb0) * (ZP * 32) + lane;
+        const uint4 zh = zp[0];
+        uint4 zl = make_uint4(0u, 0u, 0u, 0u);
+        if (ZP == 2) zl = zp[32];
+        const uint32_t st = ring_s + (uint32_t)slot * stage_bytes + lane_off;
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+            if (chunk_on[ch]) {
+                const uint32_t a = st + (uint32_t)cb[ch] * 16u;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b0, b1, b2, b3, a + (uint32_t)j * 32u);
+                    mma_bf16(acc[ch][2 * j], zh, b0, b1);
+                    mma_bf16(acc[ch][2 * j + 1], zh, b2, b3);
+                    if (ZP == 2) {
+                        mma_bf16(acc[ch][2 * j], zl, b0, b1);
+                        mma_bf16(acc[ch][2 * j + 1], zl, b2, b3);
+                    }
+                }
+            }
+        }
+        if (++slot == NS) slot = 0;
+    }
+    cp_async_wait_pending(0);
+    __syncthreads();                // the ring is idle from here on: it takes the logits and the epilogue's lists
+
+    // ---- the slab's logits to shared memory, [MT][lpitch].  Unit e of chunk ch exists if
+    // cb[ch] + e < my_units; its columns 2 t, 2 t + 1 are values (0, 1) of the tile for row g and
+    // (2, 3) for row g + 8.
+    const int lpitch = pitch * 8 + 8;
+    float* lg = reinterpret_cast<float*>(ring);
+#pragma unroll
+    for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            if (chunk_on[ch] && cb[ch] + e < my_units) {
+                float* dst = lg + (size_t)g * lpitch + (cb[ch] + e) * 8 + 2 * t;
+                if (MT == 8) {
+                    *reinterpret_cast<float2*>(dst) = make_float2(acc[ch][e][0] + acc[ch][e][2], acc[ch][e][1] + acc[ch][e][3]);
+                } else {
+                    *reinterpret_cast<float2*>(dst) = make_float2(acc[ch][e][0], acc[ch][e][1]);
+                    *reinterpret_cast<float2*>(dst + (size_t)8 * lpitch) = make_float2(acc[ch][e][2], acc[ch][e][3]);
+                }
+            }
+        }
+    __syncthreads();
+    unsigned char* lists = reinterpret_cast<unsigned char*>(lg + (size_t)MT * lpitch);
+    slab_epilogue<MT>(p, smem, lists, zarea, lg, 1, 0, lpitch, my_units * 8, unit0 * 8);
+}
+
+// ------------------------------------------------------------------------------------------
 struct Geometry {
-    int ncta, units_base, units_rem, pass_units, ct, rg, u, kc, rec_words, merge_rows, threads;
-    size_t smem;
+    int fma;             // 1: the FMA kernel (M <= 2), 0: the tensor-core kernel
+    int ncta, units_base, units_rem, rec_words;
+    int ct, rg;                                              // FMA kernel
+    int nch, pitch_units, ns, nkb, kb_chunk, nchunks;        // tensor-core kernel
+    size_t zarea_bytes, smem;
 };
 
-static bool geometry(int mt, int K, int V, int k, int sm_count, Geometry* g)
+static constexpr size_t kHeadSmemMax = 226 * 1024;
+
+static size_t merge_bytes(int) { return (size_t)(16 + 2 * 16 * 32 + 16 * 2 * kMergeCand) * 4; }
+
+// zparts: 1 or 2 parts of code fragments (tensor-core kernel)
+static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, bool want_fma, Geometry* g)
 {
-    if (V % 8 != 0 || K < 1 || k > 32 || k < 1) return false;
+    if (V % 8 != 0 || K < 1 || k > 32 || k < 1 || M < 1 || M > 16) return false;
     const int units = V / 8;
-    int ncta = sm_count < kMaxCtas ? sm_count : kMaxCtas;
+    int ncta = sm_count;
     if (ncta > units) ncta = units;
+    if (ncta > kMaxRecords) ncta = kMaxRecords;
     g->ncta = ncta;
     g->units_base = units / ncta;
     g->units_rem = units % ncta;
     const int max_units = g->units_base + (g->units_rem ? 1 : 0);
-    const int npass = (max_units + kMaxColThreads - 1) / kMaxColThreads;
-    g->pass_units = (max_units + npass - 1) / npass;
-    g->ct = (g->pass_units + 31) / 32 * 32;
-    const int nt_max = mt <= 4 ? 512 : 256;
-    g->rg = nt_max / g->ct;
-    if (g->rg < 1) g->rg = 1;
-    if (g->rg > K) g->rg = K;
-    g->threads = g->ct * g->rg;
-    g->u = (mt == 4) ? 8 : 16;
-    // rows of the code per shared-memory chunk: all of K if it fits, else a multiple of rg*u
-    const int kc_max = kZChunkBytes / (mt * 8);
-    if (K <= kc_max) g->kc = K;
-    else {
-        g->kc = kc_max / (g->rg * g->u) * (g->rg * g->u);
-        if (g->kc < 1) return false;
-    }
     g->rec_words = (2 + 2 * k + 3) / 4 * 4;
-    const size_t fixed = 128 + 16 * 64 * 4 + (size_t)mt * kMaxColWarps * 66 * 4;
-    const size_t work = (size_t)g->threads * mt * 32 + (size_t)g->kc * mt * 8;
-    const size_t one_row = (size_t)ncta * g->rec_words * 4;
-    const size_t area = work > one_row ? work : one_row;
-    g->merge_rows = (int)(area / one_row);
-    if (g->merge_rows > g->threads / 32) g->merge_rows = g->threads / 32;
-    // the first merge level parks rows * groups lists of 32 (key, id) pairs where the warps' records were
-    const int groups = (ncta + 31) / 32;
-    const int park = (int)((size_t)mt * kMaxColWarps * 66 * 4 / ((size_t)groups * 32 * 8));
-    if (park < 1) return false;
-    if (g->merge_rows > park) g->merge_rows = park;
-    g->smem = fixed + area;
-    return g->smem <= 200 * 1024;
+    const size_t fixed0 = ((kEpFixedBytes + 127) / 128) * 128;
+    g->fma = 0;
+    if (want_fma && M <= 2 && max_units <= kHeadThreads) {
+        const int mt = M;
+        g->ct = max_units;
+        int rg = kHeadThreads / g->ct;
+        if (rg > 16) rg = 16;
+        if (rg > K) rg = K;
+        g->rg = rg;
+        g->zarea_bytes = ((size_t)K * mt * 8 + 127) / 128 * 128;
+        const size_t red = (size_t)rg * mt * g->ct * 8 * 4;
+        const size_t cand = (size_t)mt * kCand * 8;
+        size_t rest = red + cand;
+        if (g->zarea_bytes + rest < merge_bytes(ncta)) rest = merge_bytes(ncta) - g->zarea_bytes;
+        g->smem = fixed0 + g->zarea_bytes + rest;
+        if (g->zarea_bytes <= kFmaCodeBytes && g->smem <= kHeadSmemMax) { g->fma = 1; return true; }
+    }
+    const int mt = M <= 8 ? 8 : 16;
+    g->nch = (max_units + 8 * kHeadWarps - 1) / (8 * kHeadWarps);
+    if (g->nch > 2) return false;
+    g->pitch_units = max_units | 1;
+    g->nkb = (K + 15) / 16;
+    const size_t kb_bytes = (size_t)zparts * 512;
+    const size_t zbytes = (size_t)g->nkb * kb_bytes;
+    if (zbytes <= kZOneChunkBytes) {
+        g->kb_chunk = g->nkb;
+        g->nchunks = 1;
+        g->zarea_bytes = zbytes;
+    } else {
+        g->kb_chunk = (int)(kZChunkBytes / kb_bytes);
+        g->nchunks = (g->nkb + g->kb_chunk - 1) / g->kb_chunk;
+        g->zarea_bytes = 2 * (size_t)g->kb_chunk * kb_bytes;
+    }
+    // the ring takes what is left; the logits, the epilogue's lists and the last CTA's merge reuse it
+    const size_t fixed = fixed0 + g->zarea_bytes + 256;
+    const size_t stage = (size_t)16 * g->pitch_units * 16;
+    const size_t ep = (size_t)mt * (g->pitch_units * 8 + 8) * 4 + (size_t)mt * kCand * 8;
+    int ns = (int)((kHeadSmemMax - fixed) / stage);
+    if (ns > kMaxStages) ns = kMaxStages;
+    if (ns < 3) return false;
+    g->ns = ns;
+    size_t ringb = (size_t)ns * stage;
+    if (ringb < ep) ringb = ep;
+    if (g->zarea_bytes + ringb < merge_bytes(ncta)) ringb = merge_bytes(ncta) - g->zarea_bytes;     // the merge works in both areas
+    g->smem = fixed + ringb;
+    return g->smem <= kHeadSmemMax;
 }
 
-StreamPlan stream_plan(int M, int d, int K, int V, int k, int sm_count)
+// The form of the code the head kernel for (M, low-rank or not) reads.
+static int code_format(const Geometry& g, int M, bool lowrank)
 {
-    StreamPlan sp = {0, 0, 0, 0};
-    (void)d;
+    if (g.fma) return kCodeF32;
+    if (!lowrank) return kCodePlain;
+    return M <= 8 ? kCodePacked : kCodeSplit;
+}
+
+StreamPlan stream_plan(int M, int K, int V, int k, int sm_count)
+{
+    StreamPlan sp = {0, 0, 0, 0, 0};
     if (M < 1) return sp;
-    const int mt = pick_mt(M > 8 ? 8 : M);
     Geometry g;
-    if (!geometry(mt, K, V, k, sm_count, &g)) return sp;
+    if (!geometry(M > 16 ? 16 : M, 2, K, V, k, sm_count, true, &g)) return sp;
     sp.ok = 1;
-    sp.mt = mt;
+    sp.mt = M <= 8 ? 8 : 16;
     sp.ncta = g.ncta;
+    sp.parts = g.ncta;
     sp.launches = 2;
     return sp;
+}
+
+size_t stream_code_bytes(int K) { return (size_t)((K + 15) / 16) * 2 * 512 + 1024; }
+
+static bool plan_code(int M, bool lowrank, int K, int V, int k, int sm_count, Geometry* g, int* fmt)
+{
+    const int zparts = (lowrank && M > 8) ? 2 : 1;
+    if (!geometry(M, zparts, K, V, k, sm_count, true, g)) return false;
+    *fmt = code_format(*g, M, lowrank);
+    return true;
 }
 
 // Launch with programmatic stream serialization: the kernel may begin once every CTA of the kernel
 // before it in the stream has signalled launch_dependents or left; it orders itself after that
 // kernel with griddepcontrol.wait.  Across calls this hides the launch gap and lets the first
 // kernel of a call warm up under the tail of the last kernel of the call before.
-template <typename... KArgs, typename... Args>
-static cudaError_t launch_early(void (*kern)(KArgs...), int grid, int block, cudaStream_t st, Args... args)
+cudaError_t stream_code(const bf16* h, const bf16* A, int M, int d, int r, int V, int k, uint32_t* zfrag, int sm_count,
+                        cudaStream_t st)
 {
+    Geometry g;
+    CodeParams cp;
+    if (!plan_code(M, true, r, V, k, sm_count, &g, &cp.fmt)) return cudaErrorInvalidValue;
+    cp.h = h; cp.A = A; cp.M = M; cp.d = d; cp.r = r; cp.zfrag = zfrag;
+    cp.nkb = (d + 15) / 16;
+    const int nct = (r + 31) / 32;
+    int S = 8;
+    while (S > 1 && (S * nct > 2 * sm_count || S * 4 > cp.nkb)) S >>= 1;
+    cp.S = S;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = 0;
+    cfg.gridDim = dim3(S, nct);
+    cfg.blockDim = dim3(128);
+    {
+        const int kbs = (cp.nkb + S - 1) / S;
+        const int rows = 16 * (kbs < kCodeChunkRows / 16 ? kbs : kCodeChunkRows / 16);
+        cfg.dynamicSmemBytes = (size_t)rows * kCodePitch + 128;
+    }
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = S;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, k_stream_code, cp);
+}
+
+cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* zfrag, int sm_count, cudaStream_t st)
+{
+    Geometry g;
+    int fmt;
+    if (!plan_code(M, false, d, V, k, sm_count, &g, &fmt)) return cudaErrorInvalidValue;
+    const int nkb = (d + 15) / 16;
+    const int n = fmt == kCodeF32 ? 2 * d : nkb * 128;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((n + 255) / 256);
+    cfg.blockDim = dim3(256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+    return cudaLaunchKernelEx(&cfg, k_stream_widen, h, M, d, nkb, fmt, zfrag);
 }
 
-cudaError_t stream_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s,
-                            cudaStream_t st)
+// Once per device: load the kernels of this file and allow the head kernels their dynamic shared
+// memory, so that no call on the hot path has to (module loading allocates and may synchronise).
+template <typename Kern>
+static cudaError_t allow_smem(Kern kern)
 {
-    const int grid = r / 16;
-    switch (mt) {
-    case 1: return launch_early(k_stream_downproj<1, 1024, 8>, grid, 1024, st, h, A, M, d, r, s.z);
-    case 2: return launch_early(k_stream_downproj<2, 1024, 4>, grid, 1024, st, h, A, M, d, r, s.z);
-    case 4: return launch_early(k_stream_downproj<4, 512, 8>, grid, 512, st, h, A, M, d, r, s.z);
-    default: return launch_early(k_stream_downproj<8, 256, 8>, grid, 256, st, h, A, M, d, r, s.z);
-    }
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kHeadSmemMax);
 }
 
-cudaError_t stream_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st)
+cudaError_t stream_prepare()
 {
-    const int n = d * mt;
-    return launch_early(k_stream_widen_t, (n + 255) / 256, 256, st, h, M, mt, d, zT);
+    cudaError_t e;
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, k_stream_code)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(k_stream_code, cudaFuncAttributeMaxDynamicSharedMemorySize, kCodeChunkRows * kCodePitch + 128)) != cudaSuccess) return e;
+    if ((e = cudaFuncGetAttributes(&fa, k_stream_widen)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_fma<1>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_fma<2>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_mma<8, 1, 1>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_mma<8, 1, 2>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_mma<16, 1, 1>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_mma<16, 1, 2>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_mma<16, 2, 1>)) != cudaSuccess) return e;
+    if ((e = allow_smem(k_stream_head_mma<16, 2, 2>)) != cudaSuccess) return e;
+    return cudaSuccess;
 }
 
-template <int MT, int U>
-static cudaError_t launch_head(const HeadParams& hp, const Geometry& g, bool pdl, cudaStream_t st)
+template <typename Kern>
+static cudaError_t launch_head(Kern kern, const HeadParams& hp, const Geometry& g, bool pdl, cudaStream_t st)
 {
-    auto kern = k_stream_head<MT, U>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem);
-    if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(hp.ncta);
-    cfg.blockDim = dim3(g.threads);
+    cfg.blockDim = dim3(kHeadThreads);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -721,31 +1164,42 @@ static cudaError_t launch_head(const HeadParams& hp, const Geometry& g, bool pdl
     return cudaLaunchKernelEx(&cfg, kern, hp);
 }
 
-cudaError_t stream_head(const float* zT, const bf16* B, int M, int mt, int K, int V, int k, int mode,
+cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int M, int K, int V, int k, int mode,
                         int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
                         bool after_producer_kernel, cudaStream_t st)
 {
     Geometry g;
-    if (!geometry(mt, K, V, k, sm_count, &g)) return cudaErrorInvalidValue;
+    int fmt;
+    if (!plan_code(M, lowrank, K, V, k, sm_count, &g, &fmt)) return cudaErrorInvalidValue;
     if (g.ncta > s.max_parts) return cudaErrorInvalidValue;
     HeadParams hp;
-    hp.zT = zT; hp.B = B; hp.M = M; hp.K = K; hp.V = V; hp.k = k; hp.mode = mode;
-    hp.ncta = g.ncta; hp.units_base = g.units_base; hp.units_rem = g.units_rem; hp.pass_units = g.pass_units;
-    hp.ct = g.ct; hp.rg = g.rg; hp.kc = g.kc; hp.rec_words = g.rec_words; hp.merge_rows = g.merge_rows;
+    memset(&hp, 0, sizeof(hp));
+    hp.zfrag = zfrag; hp.B = B; hp.M = M; hp.K = K; hp.V = V; hp.k = k; hp.mode = mode;
+    hp.ncta = g.ncta; hp.units_base = g.units_base; hp.units_rem = g.units_rem;
+    hp.rec_words = g.rec_words;
+    hp.zarea_bytes = (unsigned int)g.zarea_bytes;
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     hp.wait_prev = after_producer_kernel ? 1 : 0;
     {
-        const size_t row_bytes = (size_t)g.pass_units * 16 * g.ncta;      // one row of every slab's first pass
-        const size_t rows = row_bytes ? kPrefetchBytes / row_bytes : 0;
+        const size_t row_bytes = (size_t)V * sizeof(bf16);
+        const size_t rows = kPrefetchBytes / row_bytes;
         hp.pf_rows = after_producer_kernel ? (int)(rows < (size_t)K ? rows : (size_t)K) : 0;
     }
-    switch (mt) {
-    case 1: return launch_head<1, 16>(hp, g, after_producer_kernel, st);
-    case 2: return launch_head<2, 16>(hp, g, after_producer_kernel, st);
-    case 4: return launch_head<4, 8>(hp, g, after_producer_kernel, st);
-    default: return launch_head<8, 16>(hp, g, after_producer_kernel, st);
+    const bool pdl = after_producer_kernel;
+    if (g.fma) {
+        hp.ct = g.ct; hp.rg = g.rg;
+        const int first = g.rg * kFmaLoads < K ? g.rg * kFmaLoads : K;      // rows the kernel loads itself before it waits
+        if (hp.pf_rows > K - first) hp.pf_rows = K - first;
+        return M == 1 ? launch_head(k_stream_head_fma<1>, hp, g, pdl, st) : launch_head(k_stream_head_fma<2>, hp, g, pdl, st);
     }
+    hp.pitch_units = g.pitch_units; hp.ns = g.ns;
+    hp.nkb = g.nkb; hp.kb_chunk = g.kb_chunk; hp.nchunks = g.nchunks;
+    if (fmt == kCodeSplit)
+        return g.nch == 1 ? launch_head(k_stream_head_mma<16, 2, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 2, 2>, hp, g, pdl, st);
+    if (M <= 8)
+        return g.nch == 1 ? launch_head(k_stream_head_mma<8, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<8, 1, 2>, hp, g, pdl, st);
+    return g.nch == 1 ? launch_head(k_stream_head_mma<16, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 1, 2>, hp, g, pdl, st);
 }
 
 }  // namespace slimspec
