@@ -22,8 +22,11 @@
 
 namespace slimspec {
 
-static constexpr int kHeadWarps = 14;                 // warps of a head CTA: 64 columns each per pass
+static constexpr int kHeadWarps = 14;                 // warps of a CTA of the FMA kernel (one CTA per SM)
 static constexpr int kHeadThreads = kHeadWarps * 32;
+static constexpr int kMmaWarps = 7;                   // warps of a CTA of the tensor-core kernel (two CTAs per SM): 64 columns each
+static constexpr int kMmaThreads = kMmaWarps * 32;
+static constexpr size_t kMmaSmem = 80 * 1024;         // its shared memory: two such CTAs and the down-projection's CTA of the next call share an SM
 static constexpr int kMaxStages = 8;                  // most stages of the shared-memory ring
 static constexpr int kCand = 256;                     // candidates one row may park in a CTA's epilogue
 static constexpr int kMergeCand = 128;                // candidates one row may park in the final merge
@@ -31,18 +34,12 @@ static constexpr int kMergeLists = 10;                // slab records a lane own
 static constexpr int kMaxRecords = 32 * kMergeLists;  // records per row the merge can take
 static constexpr int kNoId = 0x7fffffff;
 enum : int { kCodeF32 = 0, kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3 };
-static constexpr size_t kZOneChunkBytes = 48 * 1024;  // code fragments up to this size stay whole in shared memory
-static constexpr size_t kZChunkBytes = 32 * 1024;     // else they pass through two buffers of this size
+static constexpr size_t kZOneChunkBytes = 16 * 1024;  // code fragments up to this size stay whole in shared memory
+static constexpr size_t kZChunkBytes = 8 * 1024;      // else they pass through two buffers of this size
 static constexpr int kEpFixedBytes = 64 + (16 * 64 + 16 + 16 + 16 + 16 * 16) * 4;
 static constexpr int kFmaLoads = 16;                  // 16-byte loads a thread of the FMA kernel keeps in flight
 static constexpr size_t kFmaCodeBytes = 64 * 1024;    // most shared memory the FMA kernel spends on the code
-
-// Bytes of the weight matrix (all CTAs together) the head kernel asks into the L2 while it waits
-// for the code: about what HBM delivers in that wait (measured; more only evicts what is needed).
-#ifndef SLIMSPEC_PF_MB
-#define SLIMSPEC_PF_MB 40
-#endif
-static constexpr size_t kPrefetchBytes = (size_t)SLIMSPEC_PF_MB << 20;
+static constexpr size_t kFmaSmem = 158 * 1024;        // its shared memory in all: the down-projection's CTA of the next call must fit beside it
 
 struct HeadParams {
     const uint32_t* zfrag;    // code: fragments [nkb][ZP][32 lanes][4 words], or fp32 [K][2] for the FMA kernel
@@ -56,6 +53,7 @@ struct HeadParams {
     int kb_chunk, nchunks;    // blocks of code fragments per shared-memory chunk, chunks
     unsigned int zarea_bytes; // shared memory the code takes
     int ct, rg;               // FMA kernel: column threads (one per unit of the widest slab) and row groups
+    int srows;                // FMA kernel: rows of the slab fetched into shared memory ahead of the code
     int rec_words;            // words per record: max, sum-exp, k (key, id) pairs, padded to 4
     int32_t* ids;
     float* logprobs;
@@ -64,7 +62,6 @@ struct HeadParams {
     unsigned int* ticket;
     int* err;
     int wait_prev;            // 1: the code is written by the kernel launched just before (PDL)
-    int pf_rows;              // rows of the slab asked into the L2 before that kernel is waited for
 };
 
 // ------------------------------------------------------------------------------------------
@@ -676,42 +673,29 @@ __device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char
     if (tid == 0) *p.ticket = 0;
 }
 
-// Common prologue of the head kernels: let the next kernel come up, ask the L2 for the first rows
-// of the slab, then wait for the kernel that writes the code.
-__device__ __forceinline__ void head_prologue(const HeadParams& p, const char* slab, int my_units, size_t Vb)
-{
-    pdl_launch_dependents();
-    if (p.wait_prev) {
-        // Until the code is there this CTA can only wait, and while it waits HBM would idle: ask the
-        // L2 for the first rows of the slab (a hint: no value is read before the wait, so whatever
-        // precedes this call in the stream may still be writing its results).
-        if (p.pf_rows > 0 && my_units > 0) {
-            const int seg_bytes = my_units * 16;
-            const int lines = (seg_bytes + 127) / 128 + 1;          // the row segment need not start on a line
-            for (int i = threadIdx.x; i < p.pf_rows * lines; i += blockDim.x) {
-                const int r = i / lines, l = i - r * lines;
-                prefetch_l2(slab + (size_t)r * Vb + min(l * 128, seg_bytes - 1));
-            }
-        }
-        pdl_wait();
-    }
-}
-
 // ------------------------------------------------------------------------------------------
 // One or two rows.  One CTA per V slab; thread = (column unit of 8 columns, row group).  Every
 // thread keeps 16 loads of its unit in flight (rows g, g + RG, g + 2 RG, ...) in two alternating
 // register sets, so that a wait for the older set never waits for loads issued after it,
 // multiplies each arriving row by the code held in shared memory as (z, z) pairs (packed FP32
 // FMAs) and refills.  The row groups' partial sums meet in shared memory.
+// While the code is not there yet (the kernel comes up early, under the tail of the call before),
+// HBM would idle: the first `srows` rows of the slab are fetched into shared memory (cp.async) and
+// the next 16 per thread into the registers, all before the wait; the main loop then works these
+// off together with what it streams.  (Asking the L2 for rows ahead of time instead was measured
+// and gains nothing: an L2 hit is served little faster than HBM serves a miss.)
+// The weights may be read before the preceding kernel has finished because they are final before
+// the call is made (the contract of the library); only the code depends on that kernel.
 template <int MT>
 __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* zarea = smem + ((kEpFixedBytes + 127) / 128) * 128;
     float2* zs = reinterpret_cast<float2*>(zarea);              // [K][MT] (z, z) pairs
-    float* red = reinterpret_cast<float*>(zarea + p.zarea_bytes);   // [RG][MT][lpitch] partial sums, then the epilogue's lists
+    unsigned char* pre = zarea + p.zarea_bytes;                 // [srows][CT * 16]: the slab's first rows; later the partial sums
+    float* red = reinterpret_cast<float*>(pre);                 // [RG][MT][lpitch] partial sums, then the epilogue's lists
     const int tid = threadIdx.x;
-    const int CT = p.ct, RG = p.rg;
+    const int CT = p.ct, RG = p.rg, S = p.srows;
     const int g = tid / CT, c = tid - g * CT;                   // row group, column unit
     const int cta = blockIdx.x;
     const int K = p.K;
@@ -720,15 +704,14 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
     const int unit0 = cta * p.units_base + min(cta, p.units_rem);
     const char* slab = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
     const int lpitch = CT * 8;
+    const uint32_t prow = (uint32_t)CT * 16u;                   // bytes between two preloaded rows
 
     constexpr int U = kFmaLoads, UH = U / 2;
     const bool active = g < RG && c < my_units;
-    const char* base = slab + (size_t)c * 16;
+    const char* base = slab + (size_t)c * 16 + (size_t)S * Vb;  // the register pipeline starts behind the preloaded rows
+    const int KR = K - S;                                       // rows it covers
     const int stepU = RG * U;
     const uint64_t pol = policy_evict_first();
-    // The first rows of the weights go out before the kernel ahead in the stream is waited for: they
-    // are final before the call is made (the contract of the library); only the code depends on that
-    // kernel.  The rows behind them are asked into the L2 meanwhile.
     uint4 q[2][UH];
     if (active) {
 #pragma unroll
@@ -736,12 +719,18 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
 #pragma unroll
             for (int j = 0; j < UH; ++j) {
                 const int row = g + (hh * UH + j) * RG;
-                q[hh][j] = row < K ? ldg_stream(base + (size_t)row * Vb, pol) : make_uint4(0u, 0u, 0u, 0u);
+                q[hh][j] = row < KR ? ldg_stream(base + (size_t)row * Vb, pol) : make_uint4(0u, 0u, 0u, 0u);
             }
     }
-    head_prologue(p, slab + (size_t)min(K, stepU) * Vb, my_units, Vb);
+    for (int idx = tid; idx < S * my_units; idx += blockDim.x) {
+        const int row = idx / my_units, cc = idx - row * my_units;
+        cp_async16(pre + (size_t)row * prow + (size_t)cc * 16, slab + (size_t)row * Vb + (size_t)cc * 16);
+    }
+    cp_async_commit();
+    pdl_launch_dependents();
+    if (p.wait_prev) pdl_wait();
     for (int i = tid; i < 16 * 64; i += blockDim.x) reinterpret_cast<float*>(smem + 64)[i] = -FLT_MAX;
-    // the code first (the main loop cannot start without it): fp32 [K][2] in global memory -> (z, z) pairs
+    // the code: fp32 [K][2] in global memory -> (z, z) pairs
     {
         const float* zf = reinterpret_cast<const float*>(p.zfrag);
         for (int e = tid; e < K * MT; e += blockDim.x) {
@@ -750,6 +739,7 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
             zs[e] = make_float2(zv, zv);
         }
     }
+    cp_async_wait_pending(0);
     __syncthreads();
 
     float2 acc[MT][4];
@@ -757,38 +747,48 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
     for (int m = 0; m < MT; ++m)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[m][e] = make_float2(0.f, 0.f);
+    auto fma_row = [&](const uint4& w4, int zrow) {
+        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+        float2 b2[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) b2[e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
+        const float2* zr = zs + (size_t)zrow * MT;
+#pragma unroll
+        for (int m = 0; m < MT; ++m) {
+            const float2 z2 = zr[m];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[m][e] = __ffma2_rn(b2[e], z2, acc[m][e]);
+        }
+    };
     if (active) {
-        for (int row = g; row < K; row += stepU) {
-            const bool checked = row - g + 2 * stepU > K;       // this block or its refills reach past K
+        // preloaded rows of this thread: g, g + RG, ... below S, a few per block of streamed rows
+        int srow = g;
+        const int nblocks = (KR + stepU - 1) / stepU;
+        const int mine = (S - g + RG - 1) / RG;
+        const int per_block = nblocks > 0 ? (mine + nblocks - 1) / nblocks : mine;
+        const unsigned char* pcol = pre + (size_t)c * 16;
+        for (int row = g; row < KR; row += stepU) {
+            const bool checked = row - g + 2 * stepU > KR;       // this block or its refills reach past the end
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
 #pragma unroll
                 for (int j = 0; j < UH; ++j) {
                     const int rj = row + (hh * UH + j) * RG;
-                    if (!checked || rj < K) {
-                        const uint32_t w[4] = {q[hh][j].x, q[hh][j].y, q[hh][j].z, q[hh][j].w};
-                        float2 b2[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            b2[e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
-                        const float2* zr = zs + (size_t)rj * MT;
-#pragma unroll
-                        for (int m = 0; m < MT; ++m) {
-                            const float2 z2 = zr[m];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) acc[m][e] = __ffma2_rn(b2[e], z2, acc[m][e]);
-                        }
-                    }
+                    if (!checked || rj < KR) fma_row(q[hh][j], S + rj);
                 }
                 // the set is used up: refill all of it at once
 #pragma unroll
                 for (int j = 0; j < UH; ++j) {
                     const int nr = row + (hh * UH + j) * RG + stepU;
-                    if (!checked || nr < K) q[hh][j] = ldg_stream(base + (size_t)nr * Vb, pol);
+                    if (!checked || nr < KR) q[hh][j] = ldg_stream(base + (size_t)nr * Vb, pol);
                 }
             }
+            for (int i = 0; i < per_block && srow < S; ++i, srow += RG)
+                fma_row(*reinterpret_cast<const uint4*>(pcol + (size_t)srow * prow), srow);
         }
+        for (; srow < S; srow += RG) fma_row(*reinterpret_cast<const uint4*>(pcol + (size_t)srow * prow), srow);
     }
+    __syncthreads();            // every thread is done with the preloaded rows: their memory takes the partial sums
     if (g < RG && c < CT) {
 #pragma unroll
         for (int m = 0; m < MT; ++m) {
@@ -803,9 +803,12 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
 }
 
 // ------------------------------------------------------------------------------------------
-// Three to sixteen rows.  One CTA per V slab, 14 warps.  The slab's rows arrive through a ring
+// Three to sixteen rows.  One CTA per V slab, seven warps, two CTAs per SM: all warps of a CTA meet
+// at a barrier once per stage and then issue their tensor-core instructions together, so a second,
+// independent CTA on the SM keeps the tensor pipe and the memory system busy meanwhile (one CTA of
+// 14 warps spent as long at the barrier as in the instructions).  The slab's rows arrive through a ring
 // of shared-memory stages (16 rows of the matrix each), filled by cp.async.  A warp owns 64 columns
-// of the slab (two such chunks when the slab is wider than 14 x 64 columns) and all K rows: per
+// of the slab (two such chunks when the slab is wider than 7 x 64 columns) and all K rows: per
 // stage it reads the "B" fragments of eight m16n8k16 instructions per chunk with ldmatrix.trans
 // (the row pitch is an odd number of 16-byte units, so the eight rows of a matrix fall into
 // distinct banks) and the code fragment from its own area of shared memory.  Lane (g, t) ends up
@@ -813,7 +816,7 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
 // of its chunks.  MT = 8: rows 8-15 of the code fragment are the remainders of rows 0-7 (or zero),
 // and the two halves of the result are summed.
 template <int MT, int ZP, int NCH>
-__global__ void __launch_bounds__(512, 1) k_stream_head_mma(const HeadParams p)      // 512: at most 128 registers, so that a small CTA fits beside it
+__global__ void __launch_bounds__(256, 2) k_stream_head_mma(const HeadParams p)      // at most 128 registers: a small CTA fits beside two of these
 {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* zarea = smem + ((kEpFixedBytes + 127) / 128) * 128;
@@ -829,7 +832,7 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_mma(const HeadParams p) 
     const int unit0 = cta * p.units_base + min(cta, p.units_rem);
     const char* slab = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
 
-    head_prologue(p, slab, my_units, Vb);
+    pdl_launch_dependents();
     for (int i = tid; i < 16 * 64; i += blockDim.x) reinterpret_cast<float*>(smem + 64)[i] = -FLT_MAX;
 
     // ---- this thread's share of a stage: 16-byte pieces (row, unit), the same for every stage
@@ -894,13 +897,18 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_mma(const HeadParams p) 
 #pragma unroll
             for (int c = 0; c < 4; ++c) acc[ch][e][c] = 0.f;
 
-    // ---- the pipeline: NS - 1 stages in flight
+    // ---- the pipeline: NS - 1 stages in flight.  The first stages go out before the kernel ahead in
+    // the stream is waited for (weights are final before the call is made: the contract of the
+    // library); the code, which that kernel writes, after it -- it travels with stage NS - 2.
+    for (int s = 0; s < NS - 2; ++s) { issue_stage(s, s); cp_async_commit(); }
+    if (p.wait_prev) pdl_wait();
     copy_zchunk(0);
-    for (int s = 0; s < NS - 1; ++s) { issue_stage(s, s); cp_async_commit(); }
+    issue_stage(NS - 2, NS - 2);
+    cp_async_commit();
     int slot = 0, fill_slot = NS - 1;
     int zc = 0, zkb0 = 0, zkb1 = min(nkb, p.kb_chunk);      // current chunk of the code
     for (int kb = 0; kb < nkb; ++kb) {
-        cp_async_wait_pending(NS - 2);
+        cp_async_wait_pending(kb == 0 ? 0 : NS - 2);        // the first time round the code, which went out last, must be in too
         __syncthreads();            // stage kb has landed for everyone; everyone is done with stage kb - 1
         if (kb == zkb1) { ++zc; zkb0 = zkb1; zkb1 = min(nkb, zkb0 + p.kb_chunk); }
         if (kb == zkb0 && p.nchunks > 1) copy_zchunk(zc + 1);
@@ -964,7 +972,7 @@ __global__ void __launch_bounds__(512, 1) k_stream_head_mma(const HeadParams p) 
 struct Geometry {
     int fma;             // 1: the FMA kernel (M <= 2), 0: the tensor-core kernel
     int ncta, units_base, units_rem, rec_words;
-    int ct, rg;                                              // FMA kernel
+    int ct, rg, srows;                                       // FMA kernel
     int nch, pitch_units, ns, nkb, kb_chunk, nchunks;        // tensor-core kernel
     size_t zarea_bytes, smem;
 };
@@ -1000,13 +1008,28 @@ static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, bool 
         const size_t cand = (size_t)mt * kCand * 8;
         size_t rest = red + cand;
         if (g->zarea_bytes + rest < merge_bytes(ncta)) rest = merge_bytes(ncta) - g->zarea_bytes;
-        g->smem = fixed0 + g->zarea_bytes + rest;
+        // what is left up to kFmaSmem holds the slab's first rows (the area is reused afterwards)
+        const size_t used = fixed0 + g->zarea_bytes;
+        const size_t prow = (size_t)g->ct * 16;
+        int srows = used + rest < kFmaSmem ? (int)((kFmaSmem - used) / prow) : (int)(rest / prow);
+        if (srows > K) srows = K;
+        g->srows = srows;
+        if ((size_t)srows * prow > rest) rest = (size_t)srows * prow;
+        g->smem = used + rest;
         if (g->zarea_bytes <= kFmaCodeBytes && g->smem <= kHeadSmemMax) { g->fma = 1; return true; }
     }
     const int mt = M <= 8 ? 8 : 16;
-    g->nch = (max_units + 8 * kHeadWarps - 1) / (8 * kHeadWarps);
+    // the tensor-core kernel: two CTAs per SM
+    ncta = 2 * sm_count;
+    if (ncta > units) ncta = units;
+    if (ncta > kMaxRecords) ncta = kMaxRecords;
+    g->ncta = ncta;
+    g->units_base = units / ncta;
+    g->units_rem = units % ncta;
+    const int mma_units = g->units_base + (g->units_rem ? 1 : 0);
+    g->nch = (mma_units + 8 * kMmaWarps - 1) / (8 * kMmaWarps);
     if (g->nch > 2) return false;
-    g->pitch_units = max_units | 1;
+    g->pitch_units = mma_units | 1;
     g->nkb = (K + 15) / 16;
     const size_t kb_bytes = (size_t)zparts * 512;
     const size_t zbytes = (size_t)g->nkb * kb_bytes;
@@ -1023,9 +1046,9 @@ static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, bool 
     const size_t fixed = fixed0 + g->zarea_bytes + 256;
     const size_t stage = (size_t)16 * g->pitch_units * 16;
     const size_t ep = (size_t)mt * (g->pitch_units * 8 + 8) * 4 + (size_t)mt * kCand * 8;
-    int ns = (int)((kHeadSmemMax - fixed) / stage);
+    if (fixed + 3 * stage > kMmaSmem) return false;
+    int ns = (int)((kMmaSmem - fixed) / stage);
     if (ns > kMaxStages) ns = kMaxStages;
-    if (ns < 3) return false;
     g->ns = ns;
     size_t ringb = (size_t)ns * stage;
     if (ringb < ep) ringb = ep;
@@ -1153,7 +1176,7 @@ static cudaError_t launch_head(Kern kern, const HeadParams& hp, const Geometry& 
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(hp.ncta);
-    cfg.blockDim = dim3(kHeadThreads);
+    cfg.blockDim = dim3(g.fma ? kHeadThreads : kMmaThreads);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -1181,16 +1204,9 @@ cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int 
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     hp.wait_prev = after_producer_kernel ? 1 : 0;
-    {
-        const size_t row_bytes = (size_t)V * sizeof(bf16);
-        const size_t rows = kPrefetchBytes / row_bytes;
-        hp.pf_rows = after_producer_kernel ? (int)(rows < (size_t)K ? rows : (size_t)K) : 0;
-    }
     const bool pdl = after_producer_kernel;
     if (g.fma) {
-        hp.ct = g.ct; hp.rg = g.rg;
-        const int first = g.rg * kFmaLoads < K ? g.rg * kFmaLoads : K;      // rows the kernel loads itself before it waits
-        if (hp.pf_rows > K - first) hp.pf_rows = K - first;
+        hp.ct = g.ct; hp.rg = g.rg; hp.srows = g.srows;
         return M == 1 ? launch_head(k_stream_head_fma<1>, hp, g, pdl, st) : launch_head(k_stream_head_fma<2>, hp, g, pdl, st);
     }
     hp.pitch_units = g.pitch_units; hp.ns = g.ns;
