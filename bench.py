@@ -38,10 +38,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture on this workload, see profiles/stream_head_c1_m1.md), keyed by the SHA-256 of the kernel's source
+# capture on this workload, see profiles/stream_head_fma_c1_m1.md), keyed by the SHA-256 of the kernel's source
 # file at the time of the capture: a changed source reports null.
 KNOWN_TRAFFIC = {
-    "cfbde1193c19711c3db3da0f6370bdaf7ed317b24a4a363a8000c6788e69bfac": 131.41e6 + 3.36e6,
 }
 
 
@@ -200,6 +199,9 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- our arm
 
+NOMINAL_HBM_GBS = 8000.0             # B200 HBM3e, nominal: reported beside the measured copy bandwidth
+
+
 def time_calls(torch, fn, n):
     """CUDA-event time of n back-to-back calls on the current stream, in milliseconds."""
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -210,6 +212,16 @@ def time_calls(torch, fn, n):
     e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1)
+
+
+def time_stats(torch, fn, n, groups=10):
+    """n calls timed as `groups` event pairs (each around n // groups back-to-back calls):
+    microseconds per call as (median, min, max) over the groups."""
+    per = max(1, n // groups)
+    vals = []
+    for g in range(groups):
+        vals.append(time_calls(torch, lambda i: fn(g * per + i), per) * 1e3 / per)
+    return {"median": statistics.median(vals), "min": min(vals), "max": max(vals), "calls": per * groups}
 
 
 def max_over_ranks(dist, ms, device):
@@ -229,6 +241,41 @@ def job_us_per_call(ms_max, steps, world):
 
 def copies_needed(nbytes):
     return max(2, -(-4 * L2_BYTES // nbytes))
+
+
+def clock_sample(gpu_index):
+    """One read-only nvidia-smi query of the SM clock and the throttle reasons (changes nothing)."""
+    try:
+        out = subprocess.run(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + ClockSampler.QUERY,
+                              "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=20).stdout
+        f = [x.strip() for x in out.strip().split(",")]
+        reasons = [n for n, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9])
+                   if v.lower().startswith("active")]
+        return {"sm_mhz": float(f[1]), "sm_max_mhz": float(f[2]), "reasons": reasons}
+    except Exception:
+        return None
+
+
+def check_against_oracle(kind, x, ids, lp, k, rows):
+    """Compare a timed point's outputs with the CPU oracle on the given rows (outside any timed region).
+    Returns the largest log-prob error and whether every rule of the parity tests held."""
+    import oracle
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from parity import check_topk
+    hb = oracle.bf16_bits(x["h"])[rows]
+    if kind == "full":
+        ref = oracle.fullhead_topk(hb, oracle.bf16_bits(x["W"]), k)
+    else:
+        ref = oracle.head_topk(hb, oracle.bf16_bits(x["A"]), oracle.bf16_bits(x["B"]), k)
+    try:
+        st = check_topk(ref, ids.cpu().numpy(), lp.cpu().numpy(), rows=rows)
+        return {"rows_checked": len(rows), "max_logprob_err": st["max_lp_err"], "ok": True}
+    except AssertionError as e:
+        return {"rows_checked": len(rows), "ok": False, "why": str(e)[:120]}
+
+
+def sample_rows(M):
+    return sorted({0, M // 2, M - 1})
 
 
 def run_ours(args):
@@ -251,7 +298,7 @@ def run_ours(args):
 
     cfg = synth.CONFIGS[WORKLOAD]
     M, d, r, V, k = 1, cfg.d, cfg.r, cfg.V, cfg.k
-    ctx = binding.Context(max_M=512, max_d=8192, max_V=V, max_k=16)
+    ctx = binding.Context(max_M=512, max_d=8192, max_V=160000, max_k=16)
     x = synth.make_inputs(M, d, r, V, seed=cfg.seed)
     R = copies_needed(2 * (d * r + r * V))
     h = x["h"].to(dev)
@@ -279,6 +326,7 @@ def run_ours(args):
     for i in range(W):
         step(i)
     barrier()
+    clk_before = clock_sample(local)
     sampler.start()
     # ---- the timed region: exactly K steps
     n0 = ctx.launch_count()
@@ -298,14 +346,23 @@ def run_ours(args):
     barrier()
     e2e_ms = max_over_ranks(dist, time_calls(torch, step_host, K), dev)
     clocks = sampler.stop()
+    clk_after = clock_sample(local)
+    if clocks["samples"] == 0:
+        # the background sampler's period is longer than a short timed region: fall back on the two
+        # synchronous reads taken directly before and after it
+        got = [c for c in (clk_before, clk_after) if c]
+        if got:
+            clocks = {"sm_mhz": statistics.median([c["sm_mhz"] for c in got]), "sm_max_mhz": max(c["sm_max_mhz"] for c in got),
+                      "reasons": sorted({r_ for c in got for r_ in c["reasons"]}), "samples": len(got)}
     if ctx.last_error() != binding.OK:
         raise SystemExit("device-side wait timed out during the benchmark")
 
     us_call = job_us_per_call(ms, K, world)
     e2e_us = job_us_per_call(e2e_ms, K, world)
     kern_us = kms * 1e3 / max(kn, 1)
-    kern_bytes = 2 * r * V + 4 * r * M            # the streamed matrix and the fp32 code
+    kern_bytes = 2 * r * V + 8 * r * M            # the streamed matrix and the fp32 code
     achieved = kern_bytes / (kern_us * 1e-6) / 1e9
+    call_gbs = head_bytes(M, d, r, V, k) / (us_call * world * 1e-6) / 1e9
 
     line = {
         "metric": METRIC, "value": us_call, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -320,13 +377,16 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
-        "roofline": {"bound": "hbm", "kernel": "k_stream_head", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        "roofline": {"bound": "hbm", "kernel": "k_stream_head_fma", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": kernel_traffic(),
                      "peak_kind": "of " + peaks_kind, "bytes_per_launch": kern_bytes, "us_per_launch": kern_us,
-                     "whole_call_frac": head_bytes(M, d, r, V, k) / (us_call * world * 1e-6) / 1e9 / peaks["hbm_gbs"]},
+                     "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+                     "whole_call_frac": call_gbs / peaks["hbm_gbs"],
+                     "whole_call_frac_of_nominal_8tbs": call_gbs / NOMINAL_HBM_GBS},
     }
 
     if rank == 0 and world == 1 and not args.no_extra:
+        line["parity_check"] = check_against_oracle("low", x, ids, lp, k, [0])
         line["extra"] = extra_points(torch, ctx, synth, binding, dev, peaks)
         line["cpu_baseline"] = cpu_baseline(cfg, M)
     ctx.close()
@@ -355,49 +415,77 @@ def cpu_baseline(cfg, M):
 
 
 def extra_points(torch, ctx, synth, binding, dev, peaks):
-    """Other points of the metric, each timed cold with CUDA events: M = 8, the full-rank head, M = 512."""
+    """The other points of the metric, each timed cold with CUDA events (median / min over ten event
+    pairs), with the kernel that streams the weights timed by itself, and checked once against the
+    oracle on sampled rows: the small head, the 8B-class head at 1 / 8 / 512 rows, the
+    larger-vocabulary head at 1 / 16 rows, the full-rank baseline."""
     out = {}
-    c1, c3 = synth.CONFIGS["c1"], synth.CONFIGS["c3"]
-    d, r, V, k = c1.d, c1.r, c1.V, c1.k
-    x = synth.make_inputs(8, d, r, V, seed=c1.seed)
-    R = copies_needed(2 * (d * r + r * V))
-    As = [x["A"].to(dev).clone() for _ in range(R)]
-    Bs = [x["B"].to(dev).clone() for _ in range(R)]
+    paths = {1: "generic", 2: "stream", 3: "tensor"}
 
-    def point(M, n):
-        h = synth.make_h(M, d, c1.seed).to(dev)
-        ids = torch.empty((M, k), dtype=torch.int32, device=dev)
-        lp = torch.empty((M, k), dtype=torch.float32, device=dev)
-        fn = lambda i: ctx.slimspec_head_topk(h, As[i % R], Bs[i % R], k, out_ids=ids, out_logprobs=lp)
-        for i in range(3):
+    def timed(fn, n, byt, flo, M):
+        for i in range(5):
             fn(i)
-        us = time_calls(torch, fn, n) * 1e3 / n
-        t_hbm = head_bytes(M, d, r, V, k) / (peaks["hbm_gbs"] * 1e9)
-        t_mma = head_flops(M, d, r, V) / (peaks["bf16_tflops"] * 1e12)
-        return {"us_per_call": us, "rows_per_s": M / (us * 1e-6), "roofline_us": max(t_hbm, t_mma) * 1e6,
-                "roofline_frac": max(t_hbm, t_mma) * 1e6 / us, "bound": "hbm" if t_hbm >= t_mma else "tensor",
-                "path": {1: "generic", 2: "stream", 3: "tensor"}.get(ctx.last_path(), "?")}
+        st = time_stats(torch, fn, n)
+        ctx.kernel_timing(True)
+        for i in range(min(n, 50)):
+            fn(i)
+        kms, kn = ctx.kernel_timing_read()
+        ctx.kernel_timing(False)
+        t_hbm = byt / (peaks["hbm_gbs"] * 1e9) * 1e6
+        t_mma = flo / (peaks["bf16_tflops"] * 1e12) * 1e6
+        roof = max(t_hbm, t_mma)
+        us = st["median"]
+        return {"us_per_call": us, "us_min": st["min"], "us_max": st["max"], "calls": st["calls"],
+                "rows_per_s": M / (us * 1e-6), "roofline_us": roof, "roofline_frac": roof / us,
+                "bound": "hbm" if t_hbm >= t_mma else "tensor",
+                "frac_of_nominal": max(byt / (NOMINAL_HBM_GBS * 1e9), flo / 2.25e15) * 1e6 / us,
+                "weights_kernel_us": kms * 1e3 / max(kn, 1), "path": paths.get(ctx.last_path(), "?")}
 
-    out["slimspec_M1"] = point(1, 200)
-    out["slimspec_M8"] = point(8, 100)
-    out["slimspec_M512"] = point(512, 20)
-    del As, Bs
+    def lowrank(name, cfgname, Ms, n_by_M, logits_too=False):
+        c = synth.CONFIGS[cfgname]
+        d, r, V, k = c.d, c.r, c.V, c.k
+        x = synth.make_inputs(max(Ms), d, r, V, seed=c.seed, logit_scale=c.logit_scale)
+        R = copies_needed(2 * (d * r + r * V))
+        As = [x["A"].to(dev).clone() for _ in range(R)]
+        Bs = [x["B"].to(dev).clone() for _ in range(R)]
+        for M in Ms:
+            xm = dict(x, h=x["h"][:M].contiguous())
+            h = xm["h"].to(dev)
+            ids = torch.empty((M, k), dtype=torch.int32, device=dev)
+            lp = torch.empty((M, k), dtype=torch.float32, device=dev)
+            fn = lambda i: ctx.slimspec_head_topk(h, As[i % R], Bs[i % R], k, out_ids=ids, out_logprobs=lp)
+            pt = timed(fn, n_by_M[M], head_bytes(M, d, r, V, k), head_flops(M, d, r, V), M)
+            torch.cuda.synchronize()
+            pt["parity_check"] = check_against_oracle("low", xm, ids, lp, k, sample_rows(M))
+            out["%s_M%d" % (name, M)] = pt
+            if logits_too:
+                lg = torch.empty((M, V), dtype=torch.float32, device=dev)
+                fl = lambda i: ctx.slimspec_head_logits(h, As[i % R], Bs[i % R], out_logits=lg)
+                out["%s_logits_M%d" % (name, M)] = timed(fl, n_by_M[M], 2 * (d * r + r * V) + 2 * M * d + 4 * M * V,
+                                                          head_flops(M, d, r, V), M)
+        del As, Bs
+
+    lowrank("c0", "c0", (1,), {1: 200}, logits_too=True)
+    lowrank("slimspec", "c1", (1, 8, 512), {1: 200, 8: 200, 512: 40})
+    lowrank("c2", "c2", (1, 16), {1: 200, 16: 200})
     # full-rank baseline: W is 1.05 GB, eight times the L2, so one copy is cold by itself
-    Wd = synth.make_W(d, V, c1.seed).to(dev)
-    for M, n in ((1, 50), (8, 20), (512, 10)):
-        h = synth.make_h(M, d, c1.seed).to(dev)
+    c1 = synth.CONFIGS["c1"]
+    d, r, V, k = c1.d, c1.r, c1.V, c1.k
+    xw = {"W": synth.make_W(d, V, c1.seed)}
+    Wd = xw["W"].to(dev)
+    for M, n in ((1, 50), (8, 50), (512, 10)):
+        hh = synth.make_h(M, d, c1.seed)
+        h = hh.to(dev)
         ids = torch.empty((M, k), dtype=torch.int32, device=dev)
         lp = torch.empty((M, k), dtype=torch.float32, device=dev)
         fn = lambda i: ctx.fullhead_topk(h, Wd, k, out_ids=ids, out_logprobs=lp)
-        for i in range(3):
-            fn(i)
-        us = time_calls(torch, fn, n) * 1e3 / n
-        fb = 2 * d * V + 2 * M * d
-        roof = max(fb / (peaks["hbm_gbs"] * 1e9), 2.0 * M * d * V / (peaks["bf16_tflops"] * 1e12)) * 1e6
-        out["fullhead_M%d" % M] = {"us_per_call": us, "roofline_us": roof, "roofline_frac": roof / us}
+        pt = timed(fn, n, fullhead_bytes(M, d, V, k), fullhead_flops(M, d, V), M)
+        torch.cuda.synchronize()
+        pt["parity_check"] = check_against_oracle("full", {"h": hh, "W": xw["W"]}, ids, lp, k, sample_rows(M)[:2])
+        out["fullhead_M%d" % M] = pt
     for M in (1, 8, 512):
         out["speedup_vs_fullhead_M%d" % M] = out["fullhead_M%d" % M]["us_per_call"] / out["slimspec_M%d" % M]["us_per_call"]
-    out["bytes_ratio_target"] = 0.8 * (d * V) / (d * r + r * V)
+    out["bytes_ratio_target"] = bytes_ratio_target(d, r, V)
     return out
 
 

@@ -21,6 +21,19 @@
  *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = the default
  *     stream) and return without synchronising, except where stated.  Calls on one
  *     context must not overlap on the GPU: a context owns one set of scratch buffers.
+ *   - Stream order, and the one exception to it.  The activations h may be produced by
+ *     whatever precedes the call in `stream`, the kernel directly before it included, and
+ *     the outputs are complete for whatever follows it.  The WEIGHTS A, B, W must be final
+ *     and visible to the device before the call is made: written by work that has completed
+ *     (a stream or event synchronisation, or work in the stream that is not still running
+ *     when the call's first kernel starts -- anything but the last kernel before the call
+ *     qualifies, and so does a memcpy).  The kernels are launched with programmatic dependent
+ *     launch and start reading weights while the kernel before the call may still be
+ *     running; a kernel that rewrites weights directly before a call (a dequantisation, a
+ *     weight swap) must be followed by an event or stream synchronisation.
+ *   - The generic path (shapes the fast kernels do not take, or forced) keeps an M x V fp32
+ *     buffer in the context for its top-k call and grows it on demand: such a call may
+ *     allocate and synchronise the device.  The fast paths never do.
  *   - Return value: SLIMSPEC_OK or a negative status; nothing is launched on an argument
  *     error.  There is no CPU fallback: every step runs in CUDA kernels.
  *   - 1 <= k <= min(V, SLIMSPEC_MAX_K).  Inputs holding NaN or infinity give unspecified
@@ -50,7 +63,7 @@ extern "C" {
 /* execution paths (slimspec_force_path) */
 #define SLIMSPEC_PATH_AUTO 0        /* chosen per (M, shapes) from measured timings            */
 #define SLIMSPEC_PATH_GENERIC 1     /* any shape; one thread per logit; slow                   */
-#define SLIMSPEC_PATH_STREAM 2      /* split-V weight-streaming kernels, FP32 FMA (small M)    */
+#define SLIMSPEC_PATH_STREAM 2      /* split-V weight-streaming kernels (M <= 16 per launch)   */
 #define SLIMSPEC_PATH_TENSOR 3      /* tcgen05 / TMEM tensor-core kernels (large M)            */
 
 typedef struct slimspec_ctx slimspec_ctx;
@@ -118,11 +131,11 @@ int slimspec_last_error(slimspec_ctx* ctx);
 long long slimspec_launch_count(const slimspec_ctx* ctx);
 
 /*
- * Device timing of the dominant kernel (the one that streams B or W), for roofline
- * reports.  While enabled, each *_topk / *_logits call records a CUDA event on its stream
- * directly before and after that kernel; the event between the down-projection and the
- * streaming kernel also keeps the two from overlapping, so the figure is the kernel alone
- * and calls are slightly slower than with timing off.  Enabling resets the totals.
+ * Device timing of the dominant kernel (the one that streams B or W, on the streaming and
+ * on the tensor-core path), for roofline reports.  While enabled, each *_topk / *_logits
+ * call records a CUDA event on its stream directly before and after that kernel; the events
+ * also keep it from overlapping its neighbours, so the figure is the kernel alone and calls
+ * are slightly slower than with timing off.  Enabling resets the totals.
  * At most 256 launches are pending at a time; the call that records the 257th first waits
  * for the earlier ones.
  */
@@ -154,8 +167,9 @@ int slimspec_kernel_timing_read(slimspec_ctx* ctx, double* total_ms, long long* 
  * SLIMSPEC_ERR_ALIGN.  h, A, B, out_ids, out_logprobs are device pointers with the layouts of
  * slimspec_head_topk; the work is enqueued on `stream` without synchronising.
  *
- * The first call on a device looks up the device address of the array (once per device, with
- * that device current); make that first call before any stream capture begins.
+ * The first call on a device looks up the device address of the array and loads the kernels
+ * (once per device, with that device current; loading is what may allocate, so it is done
+ * there and not on later calls); make that first call before any stream capture begins.
  * All calls on a device share the one array, and it keeps the previous call's contents (the
  * call clears the words that must start at zero).  Two calls whose kernels overlap on the GPU
  * -- different streams, or several host threads -- race on it: serialise them.

@@ -37,22 +37,21 @@ def build(force: bool = False) -> str:
 
 def _bind(path):
     """Load one build of the oracle and declare its signatures."""
-    if True:
-        lib = ctypes.CDLL(path)
-        u16 = ctypes.POINTER(ctypes.c_uint16)
-        f64 = ctypes.POINTER(ctypes.c_double)
-        i32 = ctypes.POINTER(ctypes.c_int32)
-        ci = ctypes.c_int
-        lib.oracle_threads.restype = ci
-        lib.oracle_set_threads.argtypes = [ci]
-        lib.oracle_downproj.argtypes = [u16, u16, ci, ci, ci, f64]
-        lib.oracle_upproj.argtypes = [f64, u16, ci, ci, ci, f64]
-        lib.oracle_slimspec_logits.argtypes = [u16, u16, u16, ci, ci, ci, ci, f64]
-        lib.oracle_slimspec_logits.restype = ci
-        lib.oracle_fullhead_logits.argtypes = [u16, u16, ci, ci, ci, f64]
-        lib.oracle_log_softmax.argtypes = [f64, ci, ci, f64, f64]
-        lib.oracle_topk.argtypes = [f64, ci, ci, ci, i32, f64, f64]
-        lib.oracle_topk.restype = ci
+    lib = ctypes.CDLL(path)
+    u16 = ctypes.POINTER(ctypes.c_uint16)
+    f64 = ctypes.POINTER(ctypes.c_double)
+    i32 = ctypes.POINTER(ctypes.c_int32)
+    ci = ctypes.c_int
+    lib.oracle_threads.restype = ci
+    lib.oracle_set_threads.argtypes = [ci]
+    lib.oracle_downproj.argtypes = [u16, u16, ci, ci, ci, f64]
+    lib.oracle_upproj.argtypes = [f64, u16, ci, ci, ci, f64]
+    lib.oracle_slimspec_logits.argtypes = [u16, u16, u16, ci, ci, ci, ci, f64]
+    lib.oracle_slimspec_logits.restype = ci
+    lib.oracle_fullhead_logits.argtypes = [u16, u16, ci, ci, ci, f64]
+    lib.oracle_log_softmax.argtypes = [f64, ci, ci, f64, f64]
+    lib.oracle_topk.argtypes = [f64, ci, ci, ci, i32, f64, f64]
+    lib.oracle_topk.restype = ci
     return lib
 
 

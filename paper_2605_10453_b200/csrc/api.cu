@@ -37,6 +37,7 @@ static const int kStreamMaxRows = 16;  // largest M the streaming path is chosen
 static const int kSplitCodeRows = 256;  // tensor path: z carried as hi + lo bf16 parts while the call is HBM-bound (up to this many rows)
 static const int kRowPad = 8;          // rows of the generic path's fp32 code are padded to this
 static const int kStreamTile = 16;     // rows one launch of the streaming kernels takes
+static const int kCodeByStreamRows = 32;   // tensor path: up to this many rows z comes from the streaming path's down-projection
 
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
@@ -281,14 +282,29 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
             // While the call is HBM-bound the tensor cores have time to spare: keep the bf16 rounding
             // remainder of z and feed it through a second MMA, so z is effectively fp32-exact.
             const bool low_part = M <= kSplitCodeRows;
-            cudaError_t e0 = tensor_downproj(h, A, M, d, r, low_part, c->s, c->sm_count, &n, st);
+            cudaError_t e0;
+            if (M <= kCodeByStreamRows && d % 2 == 0 && r % 16 == 0) {
+                // few rows: the streaming path's down-projection (one launch of small CTAs) beats a K-split
+                // tcgen05 product plus its reduction
+                e0 = stream_code_rows(h, A, M, d, r, c->s.zb, low_part ? c->s.zb_lo : (bf16*)nullptr, c->sm_count, st);
+                n = 1;
+            } else {
+                e0 = tensor_downproj(h, A, M, d, r, low_part, c->s, c->sm_count, &n, st);
+            }
             c->launches += n;
             n = 0;
             if (e0 != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
             X = c->s.zb;
             if (low_part) Xlo = c->s.zb_lo;
         }
-        cudaError_t e = tensor_head(X, Xlo, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, lowrank, &n, st);
+        if (mode == 0 && !tensor_records_fit(M, V, k, c->s, c->sm_count)) return SLIMSPEC_ERR_DIM;
+        int slot = -1;
+        if (c->timing_on) {
+            if (c->timing_used == kTimingEvents) { int rc = timing_drain(c); if (rc != SLIMSPEC_OK) return rc; }
+            slot = c->timing_used++;
+        }
+        cudaError_t e = tensor_head(X, Xlo, Bm, M, K, V, k, mode, ids, logprobs, logits, c->s, c->sm_count, &n,
+                                    slot >= 0 ? c->ev0[slot] : (cudaEvent_t) nullptr, slot >= 0 ? c->ev1[slot] : (cudaEvent_t) nullptr, st);
         c->launches += n;
         if (e != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         return SLIMSPEC_OK;

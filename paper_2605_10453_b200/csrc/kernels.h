@@ -55,6 +55,9 @@ size_t stream_code_bytes(int K);
 // code = h A for M <= 16 rows, in the form the head kernel for these shapes reads; d even, r a multiple of 16.
 cudaError_t stream_code(const bf16* h, const bf16* A, int M, int d, int r, int V, int k, uint32_t* code, int sm_count,
                         cudaStream_t st);
+// z (bf16, [M][r]) = h A and, if z_lo is not null, its rounding remainder, for any M, on the same kernel:
+// what the tensor-core path uses for small batches instead of a K-split tcgen05 product and a reduction.
+cudaError_t stream_code_rows(const bf16* h, const bf16* A, int M, int d, int r, bf16* z, bf16* z_lo, int sm_count, cudaStream_t st);
 // code = h itself (full-rank head: no down-projection).
 cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* code, int sm_count, cudaStream_t st);
 // logits = z B streamed once (M <= 16); mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
@@ -69,11 +72,12 @@ bool tensor_ok(int M, int K, int N, int k, int mode);
 cudaError_t tensor_downproj(const bf16* h, const bf16* A, int M, int d, int r, bool with_low_part, const Scratch& s,
                             int sm_count, int* launches, cudaStream_t st);
 // X W with X bf16 [M][K], W bf16 [K][N]; mode 0: fused log-softmax / top-k, mode 1: raw fp32 logits.
-// after_kernel: X is written by the kernel launched just before on `st` (the first kernel here is
-// then launched as its programmatic dependent).
 // Xlo, if not null, is added to X inside the contraction (two MMAs per step).
+// ev0 / ev1, if not null, are recorded directly before / after the kernel that streams W.
+// tensor_records_fit: does the context's record scratch take this call?
+bool tensor_records_fit(int M, int N, int k, const Scratch& s, int sm_count);
 cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
-                        float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
-                        cudaStream_t st);
+                        float* logprobs, float* logits, const Scratch& s, int sm_count, int* launches,
+                        cudaEvent_t ev0, cudaEvent_t ev1, cudaStream_t st);
 
 }  // namespace slimspec

@@ -17,6 +17,7 @@
 // K across the CTAs of a cluster and folded through distributed shared memory.
 #include "kernels.h"
 #include "ptx.cuh"
+#include "select.cuh"
 #include <float.h>
 #include <string.h>
 
@@ -29,11 +30,7 @@ static constexpr int kMmaThreads = kMmaWarps * 32;
 static constexpr size_t kMmaSmem = 80 * 1024;         // its shared memory: two such CTAs and the down-projection's CTA of the next call share an SM
 static constexpr int kMaxStages = 8;                  // most stages of the shared-memory ring
 static constexpr int kCand = 256;                     // candidates one row may park in a CTA's epilogue
-static constexpr int kMergeCand = 128;                // candidates one row may park in the final merge
-static constexpr int kMergeLists = 10;                // slab records a lane owns in the final merge
-static constexpr int kMaxRecords = 32 * kMergeLists;  // records per row the merge can take
-static constexpr int kNoId = 0x7fffffff;
-enum : int { kCodeF32 = 0, kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3 };
+enum : int { kCodeF32 = 0, kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3, kCodeRows = 4 };
 static constexpr size_t kZOneChunkBytes = 16 * 1024;  // code fragments up to this size stay whole in shared memory
 static constexpr size_t kZChunkBytes = 8 * 1024;      // else they pass through two buffers of this size
 static constexpr int kEpFixedBytes = 64 + (16 * 64 + 16 + 16 + 16 + 16 * 16) * 4;
@@ -139,93 +136,6 @@ __device__ __forceinline__ unsigned int ticket_take(unsigned int* ticket)
     return old;
 }
 
-// ------------------------------------------------------------------------------------------
-// Selection.  Candidates are (key, id) with key = f2key(logit) and key 0 = none; the order is
-// (key descending, id ascending).
-
-// The k-th largest (k = 1..32) of the warp's 32 lane values, by counting: a lane's rank is the
-// number of lanes ahead of it (larger key, or equal key and lower lane).
-__device__ __forceinline__ uint32_t warp_kth_largest(uint32_t key, int k, int lane)
-{
-    int rank = 0;
-#pragma unroll
-    for (int s = 0; s < 32; ++s) {
-        const uint32_t o = __shfl_sync(0xffffffffu, key, s);
-        rank += (o > key || (o == key && s < lane)) ? 1 : 0;
-    }
-    const unsigned hit = __ballot_sync(0xffffffffu, rank == k - 1);
-    return __shfl_sync(0xffffffffu, key, __ffs(hit) - 1);
-}
-
-// The same for small k by k rounds of "take the maximum out": cheaper than counting up to about a dozen.
-__device__ __forceinline__ uint32_t warp_kth_largest_rounds(uint32_t key, int k, int lane)
-{
-    uint32_t kth = 0u;
-    for (int j = 0; j < k; ++j) {
-        kth = warp_max_u32(key);
-        const unsigned eq = __ballot_sync(0xffffffffu, key == kth);
-        if (lane == __ffs(eq) - 1) key = 0u;
-    }
-    return kth;
-}
-__device__ __forceinline__ uint32_t warp_kth_largest_any(uint32_t key, int k, int lane)
-{
-    return k <= 12 ? warp_kth_largest_rounds(key, k, lane) : warp_kth_largest(key, k, lane);
-}
-
-// The same over 64 values, two per lane (value a has index lane, value b index lane + 32).
-__device__ __forceinline__ uint32_t warp_kth_largest64(uint32_t a, uint32_t b, int k, int lane)
-{
-    int ra = 0, rb = 0;
-#pragma unroll
-    for (int s = 0; s < 32; ++s) {
-        const uint32_t oa = __shfl_sync(0xffffffffu, a, s);
-        const uint32_t ob = __shfl_sync(0xffffffffu, b, s);
-        ra += (oa > a || (oa == a && s < lane)) ? 1 : 0;
-        ra += (ob > a) ? 1 : 0;
-        rb += (oa >= b) ? 1 : 0;
-        rb += (ob > b || (ob == b && s < lane)) ? 1 : 0;
-    }
-    const unsigned hit_a = __ballot_sync(0xffffffffu, ra == k - 1);
-    const unsigned hit_b = __ballot_sync(0xffffffffu, rb == k - 1);
-    const uint32_t va = __shfl_sync(0xffffffffu, a, hit_a ? __ffs(hit_a) - 1 : 0);
-    const uint32_t vb = __shfl_sync(0xffffffffu, b, hit_b ? __ffs(hit_b) - 1 : 0);
-    return hit_a ? va : vb;
-}
-
-// n candidates in shared memory, in any order, distinct ids.  The warp writes the min(n, k)
-// best in order to (ok, oi) and pads up to k with empty entries.  By counting: a candidate's
-// place is the number of candidates ahead of it.
-__device__ __forceinline__ void warp_rank_select(const uint32_t* ck, const int* ci, int n, int k, uint32_t* ok,
-                                                 int* oi, int lane)
-{
-    for (int base = 0; base < n; base += 32) {
-        const int i = base + lane;
-        const uint32_t mk = i < n ? ck[i] : 0u;
-        const int mi = i < n ? ci[i] : kNoId;
-        int rank = 0;
-        for (int j = 0; j < n; ++j) {
-            const uint32_t kj = ck[j];
-            const int ij = ci[j];
-            rank += (kj > mk || (kj == mk && ij < mi)) ? 1 : 0;
-        }
-        if (i < n && rank < k) { ok[rank] = mk; oi[rank] = mi; }
-    }
-    for (int j = n + lane; j < k; j += 32) { ok[j] = 0u; oi[j] = kNoId; }
-}
-
-// is (ka, ia) strictly after (kb, ib) in the order, i.e. a worse candidate?
-__device__ __forceinline__ bool after(uint32_t ka, int ia, uint32_t kb, int ib)
-{
-    return ka < kb || (ka == kb && ia > ib);
-}
-// is (ka, ia) a better candidate than (kb, ib)?
-__device__ __forceinline__ bool better(uint32_t ka, int ia, uint32_t kb, int ib)
-{
-    return ka > kb || (ka == kb && ia < ib);
-}
-
-// ------------------------------------------------------------------------------------------
 // The code z (or, for the full-rank head, h itself) reaches the head kernels in one of four forms:
 //   kCodeF32     fp32 [K][2]: entry (j, m) is z[m][j] (row 1 zero when M = 1): the FMA kernel
 //   kCodePacked  fragments, one part: rows 0-7 hold the value rounded to bf16 and rows 8-15 the
@@ -233,6 +143,8 @@ __device__ __forceinline__ bool better(uint32_t ka, int ia, uint32_t kb, int ib)
 //                (M <= 8; the two halves of its result are summed at the end)
 //   kCodeSplit   fragments, two parts: value and remainder of up to 16 rows (two instructions)
 //   kCodePlain   fragments, one part: up to 16 rows that are exact in bf16 (the full-rank head)
+//   kCodeRows    plain row-major bf16 matrices [M][r], value and remainder: the operand the tcgen05
+//                kernels load by TMA (any M: grid.z walks tiles of 16 rows)
 // Fragments: word (kb, part, lane, reg) holds, for the 16-row block kb of the streamed matrix
 // (contraction indices 16 kb .. 16 kb + 15), the two bf16 values
 //     row  = (lane >> 2) + 8 (reg & 1),   index = 16 kb + 2 (lane & 3) + 8 (reg >> 1), + 1
@@ -254,8 +166,10 @@ struct CodeParams {
     int M, d, r;
     int S;            // K splits = CTAs per cluster
     int nkb;          // 16-row blocks of A: ceil(d / 16)
-    int fmt;          // kCodeF32, kCodePacked or kCodeSplit
+    int fmt;          // kCodeF32, kCodePacked, kCodeSplit or kCodeRows
     uint32_t* zfrag;  // the code in that form
+    bf16* zrows;      // kCodeRows: value [M][r]
+    bf16* zrows_lo;   // kCodeRows: remainder [M][r], or null
 };
 
 static constexpr int kCodePitch = 80;            // bytes between two rows of the A slice in shared memory: 5 units (odd)
@@ -271,6 +185,9 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
     const int rank = blockIdx.x;
     const int j0 = blockIdx.y * 32;
     const int d = p.d, r = p.r;
+    const int m0 = blockIdx.z * 16;                      // first row of this CTA's tile of the batch
+    const int mrows = min(16, p.M - m0);
+    const bf16* hrows = p.h + (size_t)m0 * d;
     // this CTA's run of 16-row blocks, in chunks that fit the shared memory
     const int cta_kb0 = (int)((long long)p.nkb * rank / p.S), cta_kb1 = (int)((long long)p.nkb * (rank + 1) / p.S);
     auto fetch = [&](int kb0, int kb1) {
@@ -312,12 +229,12 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
                 const int k0 = 16 * (kb + i) + 2 * t;
                 const bool on = kb + i < wb1;
                 const bool lo_ok = on && k0 < d, hi_ok = on && k0 + 8 < d;
-                const uint32_t* h0 = reinterpret_cast<const uint32_t*>(p.h + (size_t)g * d + k0);
-                const uint32_t* h1 = reinterpret_cast<const uint32_t*>(p.h + (size_t)(g + 8) * d + k0);
-                hf[i].x = (g < p.M && lo_ok) ? __ldcg(h0) : 0u;
-                hf[i].y = (g + 8 < p.M && lo_ok) ? __ldcg(h1) : 0u;
-                hf[i].z = (g < p.M && hi_ok) ? __ldcg(h0 + 4) : 0u;
-                hf[i].w = (g + 8 < p.M && hi_ok) ? __ldcg(h1 + 4) : 0u;
+                const uint32_t* h0 = reinterpret_cast<const uint32_t*>(hrows + (size_t)g * d + k0);
+                const uint32_t* h1 = reinterpret_cast<const uint32_t*>(hrows + (size_t)(g + 8) * d + k0);
+                hf[i].x = (g < mrows && lo_ok) ? __ldcg(h0) : 0u;
+                hf[i].y = (g + 8 < mrows && lo_ok) ? __ldcg(h1) : 0u;
+                hf[i].z = (g < mrows && hi_ok) ? __ldcg(h0 + 4) : 0u;
+                hf[i].w = (g + 8 < mrows && hi_ok) ? __ldcg(h1 + 4) : 0u;
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
@@ -385,6 +302,14 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
         hi[e] = (uint32_t)__bfloat16_as_ushort(hb);
         lo[e] = (uint32_t)__bfloat16_as_ushort(lb);
     }
+    if (p.fmt == kCodeRows) {
+        if (row < mrows) {
+            const size_t o = (size_t)(m0 + row) * r + j;          // four bf16: 8 bytes, aligned (j is a multiple of 4)
+            *reinterpret_cast<uint2*>(p.zrows + o) = make_uint2(hi[0] | (hi[1] << 16), hi[2] | (hi[3] << 16));
+            if (p.zrows_lo) *reinterpret_cast<uint2*>(p.zrows_lo + o) = make_uint2(lo[0] | (lo[1] << 16), lo[2] | (lo[3] << 16));
+        }
+        return;
+    }
 #pragma unroll
     for (int pr = 0; pr < 2; ++pr) {
         const int jj = j + 2 * pr;
@@ -421,111 +346,6 @@ __global__ void k_stream_widen(const bf16* __restrict__ h, int M, int d, int nkb
     uint32_t word = 0u;
     if (row < M && idx < d) word = *reinterpret_cast<const uint32_t*>(h + (size_t)row * d + idx);
     zfrag[w] = word;
-}
-
-// ------------------------------------------------------------------------------------------
-// One task of the last CTA's merge, run by one warp: kind 0 = the row's log-sum-exp from the
-// records' (maximum, sum-exp) pairs, kind 1 = its k best entries.  A lane owns the records lane,
-// lane + 32, ... (NL of them at most) and keeps what it loads in registers: one round trip to the L2.
-template <int NL>
-__device__ __forceinline__ void merge_task(const HeadParams& p, int row, int kind, int lane, float* lse_s, uint32_t* ok, int* oi,
-                                           uint32_t* mk, int* mi, int* cnt)
-{
-    const int P = p.ncta, RW = p.rec_words, k = p.k;
-    const float* rows = p.part + (size_t)row * P * RW;
-    if (kind == 0) {
-        float2 ms[NL];
-#pragma unroll
-        for (int q = 0; q < NL; ++q) {
-            const int s = lane + 32 * q;
-            ms[q] = s < P ? __ldcg(reinterpret_cast<const float2*>(rows + (size_t)s * RW)) : make_float2(-FLT_MAX, 0.f);
-        }
-        float gm = -FLT_MAX;
-#pragma unroll
-        for (int q = 0; q < NL; ++q) gm = fmaxf(gm, ms[q].x);
-        gm = warp_max(gm);
-        float gs = 0.f;
-#pragma unroll
-        for (int q = 0; q < NL; ++q) gs += ms[q].y * __expf(ms[q].x - gm);
-        gs = warp_sum(gs);
-        if (lane == 0) lse_s[row] = gm + __logf(gs);
-        return;
-    }
-    // the first three entries of every record (words 2..7), then the bound: at least k entries
-    // reach the k-th largest of the lanes' best first entries
-    float2 e0[NL];
-    float4 e12[NL];
-#pragma unroll
-    for (int q = 0; q < NL; ++q) {
-        const int s = lane + 32 * q;
-        e0[q] = make_float2(0.f, __int_as_float(kNoId));
-        e12[q] = make_float4(0.f, __int_as_float(kNoId), 0.f, __int_as_float(kNoId));
-        if (s < P) {
-            e0[q] = __ldcg(reinterpret_cast<const float2*>(rows + (size_t)s * RW + 2));
-            if (k >= 2) e12[q] = __ldcg(reinterpret_cast<const float4*>(rows + (size_t)s * RW + 4));
-        }
-    }
-    uint32_t hk = 0u;
-#pragma unroll
-    for (int q = 0; q < NL; ++q) hk = max(hk, __float_as_uint(e0[q].x));
-    const uint32_t kth = warp_kth_largest_any(hk, min(k, 32), lane);
-    if (lane == 0) *cnt = 0;
-    __syncwarp();
-#pragma unroll
-    for (int q = 0; q < NL; ++q) {
-        const uint32_t k0 = __float_as_uint(e0[q].x);
-        if (k0 != 0u && k0 >= kth) {
-            int pos = atomicAdd(cnt, 1);
-            if (pos < kMergeCand) { mk[pos] = k0; mi[pos] = __float_as_int(e0[q].y); }
-            const uint32_t k1 = __float_as_uint(e12[q].x);
-            if (k >= 2 && k1 != 0u && k1 >= kth) {          // the record's list is in order: rarely more than one entry
-                pos = atomicAdd(cnt, 1);
-                if (pos < kMergeCand) { mk[pos] = k1; mi[pos] = __float_as_int(e12[q].y); }
-                const uint32_t k2 = __float_as_uint(e12[q].z);
-                if (k >= 3 && k2 != 0u && k2 >= kth) {
-                    pos = atomicAdd(cnt, 1);
-                    if (pos < kMergeCand) { mk[pos] = k2; mi[pos] = __float_as_int(e12[q].w); }
-                    const float* rec = rows + (size_t)(lane + 32 * q) * RW;
-                    for (int j = 3; j < k; ++j) {
-                        const float2 en = __ldcg(reinterpret_cast<const float2*>(rec + 2 + 2 * j));
-                        const uint32_t kj = __float_as_uint(en.x);
-                        if (kj == 0u || kj < kth) break;
-                        pos = atomicAdd(cnt, 1);
-                        if (pos < kMergeCand) { mk[pos] = kj; mi[pos] = __float_as_int(en.y); }
-                    }
-                }
-            }
-        }
-    }
-    __syncwarp();
-    const int n = *cnt;
-    if (n <= kMergeCand) {
-        warp_rank_select(mk, mi, n, k, ok, oi, lane);
-    } else {
-        // slow path: k rounds over every entry of the row's records, each round taking the best
-        // entry after the previous winner
-        uint32_t lk = 0xffffffffu;
-        int li = -1;
-        for (int j = 0; j < k; ++j) {
-            uint32_t bk = 0u;
-            int bi = kNoId;
-            for (int s = lane; s < P; s += 32) {
-                const float* rec = rows + (size_t)s * RW;
-                for (int e = 0; e < k; ++e) {
-                    const float2 en = __ldcg(reinterpret_cast<const float2*>(rec + 2 + 2 * e));
-                    const uint32_t ke = __float_as_uint(en.x);
-                    const int ie = __float_as_int(en.y);
-                    if (ke != 0u && after(ke, ie, lk, li) && better(ke, ie, bk, bi)) { bk = ke; bi = ie; }
-                }
-            }
-            const uint32_t wk = warp_max_u32(bk);
-            const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
-            lk = wk;
-            li = (int)wi;
-            if (lane == 0) { ok[j] = wk; oi[j] = wk != 0u ? (int)wi : kNoId; }
-            if (wk == 0u) { lk = 0u; li = kNoId; }
-        }
-    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -661,8 +481,8 @@ __device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char
     int* mi = reinterpret_cast<int*>(mk + kMergeCand);
     for (int task = warp; task < 2 * p.M; task += nw) {
         const int row = task >> 1;
-        if (P <= 5 * 32) merge_task<5>(p, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
-        else merge_task<kMergeLists>(p, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+        if (P <= 5 * 32) merge_task<5>(p.part, P, RW, k, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+        else merge_task<kMergeLists>(p.part, P, RW, k, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
     }
     __syncthreads();
     for (int e = tid; e < p.M * k; e += nt) {
@@ -1093,20 +913,16 @@ static bool plan_code(int M, bool lowrank, int K, int V, int k, int sm_count, Ge
 // before it in the stream has signalled launch_dependents or left; it orders itself after that
 // kernel with griddepcontrol.wait.  Across calls this hides the launch gap and lets the first
 // kernel of a call warm up under the tail of the last kernel of the call before.
-cudaError_t stream_code(const bf16* h, const bf16* A, int M, int d, int r, int V, int k, uint32_t* zfrag, int sm_count,
-                        cudaStream_t st)
+static cudaError_t launch_code(CodeParams cp, int sm_count, cudaStream_t st)
 {
-    Geometry g;
-    CodeParams cp;
-    if (!plan_code(M, true, r, V, k, sm_count, &g, &cp.fmt)) return cudaErrorInvalidValue;
-    cp.h = h; cp.A = A; cp.M = M; cp.d = d; cp.r = r; cp.zfrag = zfrag;
-    cp.nkb = (d + 15) / 16;
-    const int nct = (r + 31) / 32;
+    cp.nkb = (cp.d + 15) / 16;
+    const int nct = (cp.r + 31) / 32;
+    const int ntiles = (cp.M + 15) / 16;
     int S = 8;
     while (S > 1 && (S * nct > 2 * sm_count || S * 4 > cp.nkb)) S >>= 1;
     cp.S = S;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(S, nct);
+    cfg.gridDim = dim3(S, nct, ntiles);
     cfg.blockDim = dim3(128);
     {
         const int kbs = (cp.nkb + S - 1) / S;
@@ -1124,6 +940,27 @@ cudaError_t stream_code(const bf16* h, const bf16* A, int M, int d, int r, int V
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, k_stream_code, cp);
+}
+
+cudaError_t stream_code(const bf16* h, const bf16* A, int M, int d, int r, int V, int k, uint32_t* zfrag, int sm_count,
+                        cudaStream_t st)
+{
+    Geometry g;
+    CodeParams cp;
+    memset(&cp, 0, sizeof(cp));
+    if (!plan_code(M, true, r, V, k, sm_count, &g, &cp.fmt)) return cudaErrorInvalidValue;
+    cp.h = h; cp.A = A; cp.M = M; cp.d = d; cp.r = r; cp.zfrag = zfrag;
+    return launch_code(cp, sm_count, st);
+}
+
+cudaError_t stream_code_rows(const bf16* h, const bf16* A, int M, int d, int r, bf16* z, bf16* z_lo, int sm_count, cudaStream_t st)
+{
+    if (d % 2 != 0 || r % 16 != 0 || M < 1) return cudaErrorInvalidValue;
+    CodeParams cp;
+    memset(&cp, 0, sizeof(cp));
+    cp.fmt = kCodeRows;
+    cp.h = h; cp.A = A; cp.M = M; cp.d = d; cp.r = r; cp.zrows = z; cp.zrows_lo = z_lo;
+    return launch_code(cp, sm_count, st);
 }
 
 cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* zfrag, int sm_count, cudaStream_t st)

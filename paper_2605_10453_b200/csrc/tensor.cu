@@ -11,6 +11,7 @@
 // row and column half) and keep that row's running max / sum-exp / top-k while the next tile's MMAs run.
 #include "kernels.h"
 #include "ptx.cuh"
+#include "select.cuh"
 #include <cuda.h>
 #include <float.h>
 #include <string.h>
@@ -396,10 +397,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) k_tc_gemm(const __grid_constant
             float* rec = p.part + ((size_t)m * (2 * p.gct) + 2 * cg + half) * p.rec_words;
             rec[0] = run_max;
             rec[1] = run_sum;
-            for (int j = 0; j < k; ++j) {
-                rec[2 + j] = __uint_as_float(j < cnt ? f2key(sv[j] + 0.f) : 0u);      // -0 and +0 rank alike
-                rec[2 + k + j] = __int_as_float(j < cnt ? si[j] : kTcNoId);
-            }
+            for (int j = 0; j < k; ++j)      // (key, id) pairs; -0 and +0 rank alike
+                *reinterpret_cast<float2*>(rec + 2 + 2 * j) =
+                    make_float2(__uint_as_float(j < cnt ? f2key(sv[j] + 0.f) : 0u), __int_as_float(j < cnt ? si[j] : kTcNoId));
         }
     }
     // ---- teardown: every role is past its last use of tensor memory
@@ -457,79 +457,30 @@ __global__ void __launch_bounds__(256) k_tc_thr0(const uint32_t* __restrict__ sm
 }
 
 // ------------------------------------------------------------------------------------------
-// Merge the P per-slab records of each row: one warp per row, a lane owns up to 10 slab lists
-// and keeps each list's head and the entry after it in registers, so that a pop never waits for
-// memory unless the same list wins twice in a row.
-static constexpr int kMergeLists = 10;
-
+// Merge the P per-slab records of each row.  Two rows per CTA, two warps per row: one takes the
+// row's log-sum-exp, the other its k best entries (bound from the records' first entries, the few
+// entries above it ordered by counting).
 __global__ void __launch_bounds__(128) k_tc_merge(const float* __restrict__ part, int M, int P, int RW, int k,
                                                   int32_t* __restrict__ ids, float* __restrict__ logprobs)
 {
+    __shared__ float lse_s[2];
+    __shared__ uint32_t ok_s[2][32];
+    __shared__ int oi_s[2][32];
+    __shared__ uint32_t mk_s[4][kMergeCand];
+    __shared__ int mi_s[4][kMergeCand];
+    __shared__ int cnt_s[4];
     pdl_launch_dependents();     // the first kernel of the next call may come up behind this one
     pdl_wait();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m = blockIdx.x * (blockDim.x >> 5) + warp;
-    if (m >= M) return;
-    const float* rows = part + (size_t)m * P * RW;
-    uint32_t hk[kMergeLists], nk[kMergeLists];
-    int hi[kMergeLists], ni[kMergeLists], hp[kMergeLists];
-    float pm[kMergeLists], ps[kMergeLists];
-#pragma unroll
-    for (int q = 0; q < kMergeLists; ++q) {
-        const int s = lane + 32 * q;
-        const bool have = s < P;
-        const float* rec = rows + (size_t)(have ? s : 0) * RW;
-        hp[q] = 0;
-        pm[q] = have ? __ldcg(rec) : -FLT_MAX;
-        ps[q] = have ? __ldcg(rec + 1) : 0.f;
-        hk[q] = have ? __float_as_uint(__ldcg(rec + 2)) : 0u;
-        hi[q] = have ? __float_as_int(__ldcg(rec + 2 + k)) : kTcNoId;
-        nk[q] = (have && k > 1) ? __float_as_uint(__ldcg(rec + 3)) : 0u;
-        ni[q] = (have && k > 1) ? __float_as_int(__ldcg(rec + 3 + k)) : kTcNoId;
+    const int r2 = warp >> 1, row = blockIdx.x * 2 + r2;
+    if (row < M) {
+        if (P <= 5 * 32) merge_task<5>(part, P, RW, k, row, warp & 1, lane, lse_s - row + r2, ok_s[r2], oi_s[r2], mk_s[warp], mi_s[warp], &cnt_s[warp]);
+        else merge_task<kMergeLists>(part, P, RW, k, row, warp & 1, lane, lse_s - row + r2, ok_s[r2], oi_s[r2], mk_s[warp], mi_s[warp], &cnt_s[warp]);
     }
-    float gm = -FLT_MAX;
-#pragma unroll
-    for (int q = 0; q < kMergeLists; ++q) gm = fmaxf(gm, pm[q]);
-    gm = warp_max(gm);
-    float gs = 0.f;
-#pragma unroll
-    for (int q = 0; q < kMergeLists; ++q) gs += ps[q] * __expf(pm[q] - gm);
-    gs = warp_sum(gs);
-    const float lse = gm + __logf(gs);
-    uint32_t ok = 0;
-    int oi = kTcNoId;
-    for (int j = 0; j < k; ++j) {
-        uint32_t bk = hk[0];
-        int bi = hi[0], bs = 0;
-#pragma unroll
-        for (int q = 1; q < kMergeLists; ++q) {
-            const bool better = hk[q] > bk || (hk[q] == bk && hi[q] < bi);
-            bk = better ? hk[q] : bk;
-            bi = better ? hi[q] : bi;
-            bs = better ? q : bs;
-        }
-        const uint32_t wk = warp_max_u32(bk);
-        const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
-        const bool win = (bk == wk) && ((uint32_t)bi == wi) && wk != 0u;
-#pragma unroll
-        for (int q = 0; q < kMergeLists; ++q) {
-            if (win && q == bs) {
-                const int s = lane + 32 * q;
-                const int np = hp[q] + 1;
-                hp[q] = np;
-                hk[q] = nk[q];
-                hi[q] = ni[q];
-                const bool more = np + 1 < k;
-                const float* rec = rows + (size_t)s * RW;
-                nk[q] = more ? __float_as_uint(__ldcg(rec + 3 + np)) : 0u;
-                ni[q] = more ? __float_as_int(__ldcg(rec + 3 + k + np)) : kTcNoId;
-            }
-        }
-        if (lane == j) { ok = wk; oi = (int)wi; }
-    }
-    if (lane < k) {
-        ids[(size_t)m * k + lane] = oi;
-        logprobs[(size_t)m * k + lane] = key2f(ok) - lse;
+    __syncthreads();
+    if ((warp & 1) == 0 && row < M && lane < k) {
+        ids[(size_t)row * k + lane] = oi_s[r2][lane];
+        logprobs[(size_t)row * k + lane] = key2f(ok_s[r2][lane]) - lse_s[r2];
     }
 }
 
@@ -615,15 +566,28 @@ static cudaError_t launch_gemm(TcParams p, int grid, bool pdl, cudaStream_t st)
     return launch_chain(kern, grid, kTcThreads, smem, pdl, st, p);
 }
 
+// Does the context's scratch hold the split-V records of this call?  (Same arithmetic as tensor_head.)
+bool tensor_records_fit(int M, int N, int k, const Scratch& s, int sm_count)
+{
+    const int nrb = (M + kTcRows - 1) / kTcRows;
+    const int nv = (nrb == 1) ? 128 : 256;
+    const int nct = (N + nv - 1) / nv;
+    int gct = sm_count / nrb;
+    if (gct < 1) gct = 1;
+    if (gct > nct) gct = nct;
+    if (gct > kMaxRecords / 2) gct = kMaxRecords / 2;
+    return (size_t)M * 2 * gct * ((2 + 2 * k + 3) / 4 * 4) <= s.part_elems;
+}
+
 // out = X W through the tensor cores.  mode 0: top-k records then merge into ids / logprobs;
 // mode 1: fp32 logits.  X is bf16 [M][K], W bf16 [K][N].
 cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, int K, int N, int k, int mode, int32_t* ids,
-                        float* logprobs, float* logits, const Scratch& s, int sm_count, bool after_kernel, int* launches,
-                        cudaStream_t st)
+                        float* logprobs, float* logits, const Scratch& s, int sm_count, int* launches,
+                        cudaEvent_t ev0, cudaEvent_t ev1, cudaStream_t st)
 {
     // Every kernel here orders itself after its predecessor with griddepcontrol.wait before it touches
     // global memory, so each one, the first included, is launched early.
-    after_kernel = true;
+    const bool after_kernel = true;
     TcParams p;
     memset(&p, 0, sizeof(p));
     // a single row block loads only as many rows of X as there are (in whole groups of eight)
@@ -644,7 +608,7 @@ cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, in
     p.gct = sm_count / p.nrb;
     if (p.gct < 1) p.gct = 1;
     if (p.gct > p.nct) p.gct = p.nct;
-    if (p.gct > 160) p.gct = 160;       // the merge takes up to 320 lists per row
+    if (p.gct > kMaxRecords / 2) p.gct = kMaxRecords / 2;       // the merge takes up to 320 lists per row
     p.mode = mode;
     p.k = k;
     p.rec_words = (2 + 2 * k + 3) / 4 * 4;
@@ -672,18 +636,21 @@ cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, in
             if (e != cudaSuccess) return e;
             e = launch_chain(k_tc_thr0, (M + 7) / 8, 256, 0, true, st, (const uint32_t*)s.smax, 2 * nst, p.nrb * kTcRows, M, k,
                              s.thr0);
-            after_kernel = true;
             if (e != cudaSuccess) return e;
             *launches += 2;
             p.thr0 = s.thr0;
         }
     }
     const int grid = p.gct * p.nrb;
-    e = (nv == 128) ? launch_gemm<128>(p, grid, after_kernel, st) : launch_gemm<256>(p, grid, after_kernel, st);
+    // optional events directly around the kernel that streams the weights (they also keep it from
+    // overlapping its neighbours)
+    if (ev0 && (e = cudaEventRecord(ev0, st)) != cudaSuccess) return e;
+    e = (nv == 128) ? launch_gemm<128>(p, grid, after_kernel && !ev0, st) : launch_gemm<256>(p, grid, after_kernel && !ev0, st);
     if (e != cudaSuccess) return e;
+    if (ev1 && (e = cudaEventRecord(ev1, st)) != cudaSuccess) return e;
     *launches += 1;
     if (mode == 0) {
-        e = launch_chain(k_tc_merge, (M + 3) / 4, 128, 0, true, st, (const float*)s.part, M, 2 * p.gct, p.rec_words, k, ids,
+        e = launch_chain(k_tc_merge, (M + 1) / 2, 128, 0, true, st, (const float*)s.part, M, 2 * p.gct, p.rec_words, k, ids,
                          logprobs);
         *launches += 1;
     }

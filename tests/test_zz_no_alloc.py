@@ -61,6 +61,22 @@ def test_static_scratch_entry_point_matches_the_oracle():
         assert st["max_lp_err"] <= 1e-3
 
 
+def test_static_scratch_entry_point_allocates_nothing_after_its_first_call():
+    """One warm-up call sets the entry point up (symbol address, kernels loaded); after it, calls of
+    every row-count class leave the device's free memory unchanged."""
+    d, r, V, k = 512, 128, 8 * 1501, 7
+    xs = {M: {n: t.to(DEV) for n, t in synth.make_inputs(M, d, r, V, seed=M).items()} for M in (1, 2, 4, 8)}
+    outs = {M: (torch.empty((M, k), dtype=torch.int32, device=DEV), torch.empty((M, k), dtype=torch.float32, device=DEV))
+            for M in xs}
+    binding.slimspec_head_topk_static(xs[1]["h"], xs[1]["A"], xs[1]["B"], k, *outs[1])      # the warm-up
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for M in (1, 2, 4, 8):
+        binding.slimspec_head_topk_static(xs[M]["h"], xs[M]["A"], xs[M]["B"], k, *outs[M])
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+
+
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
     lib = binding.load()
     g = {n: t.to(DEV) for n, t in synth.make_inputs(2, 64, 64, 800, seed=1).items()}
