@@ -315,6 +315,7 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         const int mrows = (M - m0 < kStreamTile) ? (M - m0) : kStreamTile;
         const bf16* hm = h + (size_t)m0 * d;
         const int kk = mode == 0 ? k : 1;
+        int nl = 0;
         if (lowrank) CK(stream_code(hm, A, mrows, d, r, V, kk, c->s.zfrag, c->sm_count, st));
         else CK(stream_widen(hm, mrows, d, V, kk, c->s.zfrag, c->sm_count, st));
         int slot = -1;
@@ -327,9 +328,9 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         CK(stream_head(c->s.zfrag, lowrank, Bm, mrows, K, V, kk, mode,
                        mode == 0 ? ids + (size_t)m0 * k : nullptr,
                        mode == 0 ? logprobs + (size_t)m0 * k : nullptr,
-                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, slot < 0, st));
+                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, slot < 0, &nl, st));
         if (slot >= 0) CK(cudaEventRecord(c->ev1[slot], st));
-        c->launches += 2;
+        c->launches += 1 + nl;
     }
     return SLIMSPEC_OK;
 }

@@ -63,7 +63,10 @@ cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* co
 // logits = z B streamed once (M <= 16); mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
 cudaError_t stream_head(const uint32_t* code, bool lowrank, const bf16* B, int M, int K, int V, int k, int mode,
                         int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
-                        bool after_producer_kernel, cudaStream_t st);
+                        bool after_producer_kernel, int* launches, cudaStream_t st);
+
+// ---- the merge of split-V records as a kernel of its own (tensor path; streaming path with many rows)
+cudaError_t merge_records(const float* part, int M, int P, int RW, int k, int32_t* ids, float* logprobs, cudaStream_t st);
 
 // ---- tensor-core path (larger M) ------------------------------------------------------
 // Shapes the tcgen05 kernels take: K a multiple of 64, N a multiple of 8 and >= 64, k <= 32 in top-k mode.

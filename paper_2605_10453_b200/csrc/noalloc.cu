@@ -87,7 +87,7 @@ extern "C" int slimspec_head_topk_static(const void* h, const void* A, const voi
     // The array keeps whatever the last call left; the ticket and the error word must start at 0.
     if (cudaMemsetAsync(dev->base + kZBytes + kPartBytes, 0, kCtlBytes, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
     if (stream_code((const bf16*)h, (const bf16*)A, M, d, r, V, k, s.zfrag, dev->sm_count, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
-    if (stream_head(s.zfrag, true, (const bf16*)B, M, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, st) !=
+    if (stream_head(s.zfrag, true, (const bf16*)B, M, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, nullptr, st) !=
         cudaSuccess) {
         cudaGetLastError();
         return SLIMSPEC_ERR_CUDA;

@@ -22,7 +22,7 @@ static constexpr int kNoId = 0x7fffffff;
 __device__ __forceinline__ uint32_t warp_kth_largest(uint32_t key, int k, int lane)
 {
     int rank = 0;
-#pragma unroll
+#pragma unroll 4
     for (int s = 0; s < 32; ++s) {
         const uint32_t o = __shfl_sync(0xffffffffu, key, s);
         rank += (o > key || (o == key && s < lane)) ? 1 : 0;
@@ -51,7 +51,7 @@ __device__ __forceinline__ uint32_t warp_kth_largest_any(uint32_t key, int k, in
 __device__ __forceinline__ uint32_t warp_kth_largest64(uint32_t a, uint32_t b, int k, int lane)
 {
     int ra = 0, rb = 0;
-#pragma unroll
+#pragma unroll 4
     for (int s = 0; s < 32; ++s) {
         const uint32_t oa = __shfl_sync(0xffffffffu, a, s);
         const uint32_t ob = __shfl_sync(0xffffffffu, b, s);

@@ -59,6 +59,7 @@ struct HeadParams {
     unsigned int* ticket;
     int* err;
     int wait_prev;            // 1: the code is written by the kernel launched just before (PDL)
+    int merge_inside;         // 1: the last CTA to arrive merges the records; 0: the merge kernel follows
 };
 
 // ------------------------------------------------------------------------------------------
@@ -385,18 +386,32 @@ __device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char
             for (int c = tid; c < ncols; c += nt) p.logits[(size_t)row * p.V + col_base + c] = logit(row, c);
         return;
     }
-    // ---- (1)
-    for (int row = 0; row < mrows; ++row) {
-        float m = -FLT_MAX;
-        for (int c = tid; c < ncols; c += nt) m = fmaxf(m, logit(row, c));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 4));
-        if ((lane & 7) == 0) gmax_s[row * 64 + warp * 4 + (lane >> 3)] = m;
+    // ---- (1)  (rows in batches, so that their shuffle chains overlap)
+    constexpr int RB = MT < 4 ? MT : 4;
+    for (int row0 = 0; row0 < mrows; row0 += RB) {
+        float m[RB];
+#pragma unroll
+        for (int i = 0; i < RB; ++i) m[i] = -FLT_MAX;
+        for (int c = tid; c < ncols; c += nt) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i)
+                if (row0 + i < mrows) m[i] = fmaxf(m[i], logit(row0 + i, c));
+        }
+#pragma unroll
+        for (int o = 1; o <= 4; o <<= 1) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], o));
+        }
+        if ((lane & 7) == 0) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i)
+                if (row0 + i < mrows) gmax_s[(row0 + i) * 64 + warp * 4 + (lane >> 3)] = m[i];
+        }
     }
     __syncthreads();
     // ---- (2)  Up to 16 candidates wanted, the maxima of slot pairs do (32 values, half the
-    // shuffles); beyond that all 64 slots are ranked.
+    // shuffles); beyond that all 64 slots are ranked.  (Kept as one short loop: a version that ran the
+    // rounds of a warp's rows interleaved grew the kernels by 40 % and cost 2.5 us per call.)
     for (int row = warp; row < mrows; row += nw) {
         const uint32_t ka = f2key(gmax_s[row * 64 + lane]), kb2 = f2key(gmax_s[row * 64 + 32 + lane]);
         const uint32_t kth = (k <= 16) ? warp_kth_largest_any(max(ka, kb2), k, lane) : warp_kth_largest64(ka, kb2, min(k, 64), lane);
@@ -405,19 +420,37 @@ __device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char
     }
     __syncthreads();
     // ---- (3)
-    for (int row = 0; row < mrows; ++row) {
-        const float tau = tau_s[row], cm = cmax_s[row];
-        float s = 0.f;
+    for (int row0 = 0; row0 < mrows; row0 += RB) {
+        float s[RB], tau[RB], cm[RB];
+#pragma unroll
+        for (int i = 0; i < RB; ++i) {
+            const int row = min(row0 + i, mrows - 1);
+            s[i] = 0.f; tau[i] = tau_s[row]; cm[i] = cmax_s[row];
+        }
         for (int c = tid; c < ncols; c += nt) {
-            const float x = logit(row, c);
-            s += __expf(x - cm);
-            if (x >= tau) {
-                const int pos = atomicAdd(&cnt_s[row], 1);
-                if (pos < kCand) { ck[row * kCand + pos] = f2key(x); ci[row * kCand + pos] = col_base + c; }
+#pragma unroll
+            for (int i = 0; i < RB; ++i) {
+                if (row0 + i < mrows) {
+                    const int row = row0 + i;
+                    const float x = logit(row, c);
+                    s[i] += __expf(x - cm[i]);
+                    if (x >= tau[i]) {
+                        const int pos = atomicAdd(&cnt_s[row], 1);
+                        if (pos < kCand) { ck[row * kCand + pos] = f2key(x); ci[row * kCand + pos] = col_base + c; }
+                    }
+                }
             }
         }
-        s = warp_sum(s);
-        if (lane == 0) wsum_s[row * 16 + warp] = s;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i)
+                if (row0 + i < mrows) wsum_s[(row0 + i) * 16 + warp] = s[i];
+        }
     }
     __syncthreads();
     // ---- (4)
@@ -467,7 +500,9 @@ __device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char
         }
     }
 
-    // ---- arrival: the last CTA merges the records of every row
+    // ---- arrival: the last CTA merges the records of every row (many rows: a kernel of its own does,
+    // with two warps per row on as many SMs as it takes)
+    if (!p.merge_inside) return;
     __syncthreads();
     if (tid == 0) *s_ticket = ticket_take(p.ticket);
     __syncthreads();
@@ -1026,7 +1061,7 @@ static cudaError_t launch_head(Kern kern, const HeadParams& hp, const Geometry& 
 
 cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int M, int K, int V, int k, int mode,
                         int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
-                        bool after_producer_kernel, cudaStream_t st)
+                        bool after_producer_kernel, int* launches, cudaStream_t st)
 {
     Geometry g;
     int fmt;
@@ -1041,18 +1076,25 @@ cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int 
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     hp.wait_prev = after_producer_kernel ? 1 : 0;
+    hp.merge_inside = (mode == 1 || M <= 7) ? 1 : 0;       // measured: from 8 rows on the merge kernel is faster (2 us at 8 rows)
     const bool pdl = after_producer_kernel;
+    cudaError_t e;
     if (g.fma) {
         hp.ct = g.ct; hp.rg = g.rg; hp.srows = g.srows;
-        return M == 1 ? launch_head(k_stream_head_fma<1>, hp, g, pdl, st) : launch_head(k_stream_head_fma<2>, hp, g, pdl, st);
+        e = M == 1 ? launch_head(k_stream_head_fma<1>, hp, g, pdl, st) : launch_head(k_stream_head_fma<2>, hp, g, pdl, st);
+    } else {
+        hp.pitch_units = g.pitch_units; hp.ns = g.ns;
+        hp.nkb = g.nkb; hp.kb_chunk = g.kb_chunk; hp.nchunks = g.nchunks;
+        if (fmt == kCodeSplit)
+            e = g.nch == 1 ? launch_head(k_stream_head_mma<16, 2, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 2, 2>, hp, g, pdl, st);
+        else if (M <= 8)
+            e = g.nch == 1 ? launch_head(k_stream_head_mma<8, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<8, 1, 2>, hp, g, pdl, st);
+        else
+            e = g.nch == 1 ? launch_head(k_stream_head_mma<16, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 1, 2>, hp, g, pdl, st);
     }
-    hp.pitch_units = g.pitch_units; hp.ns = g.ns;
-    hp.nkb = g.nkb; hp.kb_chunk = g.kb_chunk; hp.nchunks = g.nchunks;
-    if (fmt == kCodeSplit)
-        return g.nch == 1 ? launch_head(k_stream_head_mma<16, 2, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 2, 2>, hp, g, pdl, st);
-    if (M <= 8)
-        return g.nch == 1 ? launch_head(k_stream_head_mma<8, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<8, 1, 2>, hp, g, pdl, st);
-    return g.nch == 1 ? launch_head(k_stream_head_mma<16, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 1, 2>, hp, g, pdl, st);
+    if (launches) *launches += hp.merge_inside ? 1 : 2;
+    if (e != cudaSuccess || hp.merge_inside) return e;
+    return merge_records(s.part, M, hp.ncta, hp.rec_words, k, ids, logprobs, st);
 }
 
 }  // namespace slimspec

@@ -544,6 +544,12 @@ static cudaError_t launch_chain(void (*kern)(KArgs...), int grid, int block, siz
     return cudaLaunchKernelEx(&cfg, kern, args...);
 }
 
+// Merge kernel: P split-V records per row -> ids / log-probs; launched early behind the kernel that writes them.
+cudaError_t merge_records(const float* part, int M, int P, int RW, int k, int32_t* ids, float* logprobs, cudaStream_t st)
+{
+    return launch_chain(k_tc_merge, (M + 1) / 2, 128, 0, true, st, part, M, P, RW, k, ids, logprobs);
+}
+
 // Chooses the ring depth (and whether X can stay resident) and launches.
 template <int NV>
 static cudaError_t launch_gemm(TcParams p, int grid, bool pdl, cudaStream_t st)
@@ -650,8 +656,7 @@ cudaError_t tensor_head(const bf16* X, const bf16* Xlo, const bf16* W, int M, in
     if (ev1 && (e = cudaEventRecord(ev1, st)) != cudaSuccess) return e;
     *launches += 1;
     if (mode == 0) {
-        e = launch_chain(k_tc_merge, (M + 1) / 2, 128, 0, true, st, (const float*)s.part, M, 2 * p.gct, p.rec_words, k, ids,
-                         logprobs);
+        e = merge_records(s.part, M, 2 * p.gct, p.rec_words, k, ids, logprobs, st);
         *launches += 1;
     }
     return e;
