@@ -7,7 +7,7 @@ import subprocess
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libslimspec.so")
-SOURCES = ["api.cu", "generic.cu", "stream.cu", "noalloc.cu", "tensor.cu"]
+SOURCES = ["api.cu", "generic.cu", "stream.cu", "stream_fma.cu", "noalloc.cu", "tensor.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-shared",

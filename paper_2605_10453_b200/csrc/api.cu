@@ -112,7 +112,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     ok = ok && cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.err, 0, sizeof(int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.z, 0, z_elems * sizeof(float)) == cudaSuccess;
-    ok = ok && stream_prepare() == cudaSuccess;
+    ok = ok && stream_prepare() == cudaSuccess && fma_prepare() == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -316,8 +316,16 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         const bf16* hm = h + (size_t)m0 * d;
         const int kk = mode == 0 ? k : 1;
         int nl = 0;
-        if (lowrank) CK(stream_code(hm, A, mrows, d, r, V, kk, c->s.zfrag, c->sm_count, st));
-        else CK(stream_widen(hm, mrows, d, V, kk, c->s.zfrag, c->sm_count, st));
+        // one or two rows: the FMA kernels; three to sixteen: the tensor-core streaming kernels
+        const FmaPlan fp = fma_plan(mrows, d, K, V, kk, c->sm_count);
+        const bool fma = fp.ok && fp.ncta <= c->s.max_parts;
+        if (fma) {
+            if (lowrank) CK(fma_downproj(hm, A, mrows, fp.mt, d, r, c->s, st));
+            else CK(fma_widen_t(hm, mrows, fp.mt, d, c->s.z, st));
+        } else {
+            if (lowrank) CK(stream_code(hm, A, mrows, d, r, V, kk, c->s.zfrag, c->sm_count, st));
+            else CK(stream_widen(hm, mrows, d, V, kk, c->s.zfrag, c->sm_count, st));
+        }
         int slot = -1;
         if (c->timing_on) {
             if (c->timing_used == kTimingEvents) { int rc = timing_drain(c); if (rc != SLIMSPEC_OK) return rc; }
@@ -325,10 +333,15 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
             CK(cudaEventRecord(c->ev0[slot], st));
         }
         // an event between the two kernels serialises them: the timed kernel then runs alone
-        CK(stream_head(c->s.zfrag, lowrank, Bm, mrows, K, V, kk, mode,
-                       mode == 0 ? ids + (size_t)m0 * k : nullptr,
-                       mode == 0 ? logprobs + (size_t)m0 * k : nullptr,
-                       mode == 1 ? logits + (size_t)m0 * V : nullptr, c->s, c->sm_count, slot < 0, &nl, st));
+        int32_t* ids_t = mode == 0 ? ids + (size_t)m0 * k : nullptr;
+        float* lp_t = mode == 0 ? logprobs + (size_t)m0 * k : nullptr;
+        float* lg_t = mode == 1 ? logits + (size_t)m0 * V : nullptr;
+        if (fma) {
+            CK(fma_head(c->s.z, Bm, mrows, fp.mt, K, V, kk, mode, ids_t, lp_t, lg_t, c->s, c->sm_count, slot < 0, st));
+            nl = 1;
+        } else {
+            CK(stream_head(c->s.zfrag, lowrank, Bm, mrows, K, V, kk, mode, ids_t, lp_t, lg_t, c->s, c->sm_count, slot < 0, &nl, st));
+        }
         if (slot >= 0) CK(cudaEventRecord(c->ev1[slot], st));
         c->launches += 1 + nl;
     }

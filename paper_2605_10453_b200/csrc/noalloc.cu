@@ -50,7 +50,7 @@ int setup_current_device(DeviceSetup** out)
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         // load the kernels now, so that no later call has to (loading a module allocates)
-        if (stream_prepare() != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
+        if (stream_prepare() != cudaSuccess || fma_prepare() != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
         s.base = static_cast<unsigned char*>(ptr);
         s.sm_count = sms;
         s.ready = true;
@@ -86,11 +86,17 @@ extern "C" int slimspec_head_topk_static(const void* h, const void* A, const voi
     cudaStream_t st = (cudaStream_t)stream;
     // The array keeps whatever the last call left; the ticket and the error word must start at 0.
     if (cudaMemsetAsync(dev->base + kZBytes + kPartBytes, 0, kCtlBytes, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
-    if (stream_code((const bf16*)h, (const bf16*)A, M, d, r, V, k, s.zfrag, dev->sm_count, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
-    if (stream_head(s.zfrag, true, (const bf16*)B, M, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, nullptr, st) !=
-        cudaSuccess) {
-        cudaGetLastError();
-        return SLIMSPEC_ERR_CUDA;
+    // the same choice of kernels as the context-based entry point: one or two rows, the FMA kernels
+    const FmaPlan fp = fma_plan(M, d, r, V, k, dev->sm_count);
+    cudaError_t e;
+    if (fp.ok && fp.ncta <= kStaticParts) {
+        s.z = reinterpret_cast<float*>(dev->base);          // fp32 code, [r][mt]: it fits where the fragments would go
+        e = fma_downproj((const bf16*)h, (const bf16*)A, M, fp.mt, d, r, s, st);
+        if (e == cudaSuccess) e = fma_head(s.z, (const bf16*)B, M, fp.mt, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, st);
+    } else {
+        e = stream_code((const bf16*)h, (const bf16*)A, M, d, r, V, k, s.zfrag, dev->sm_count, st);
+        if (e == cudaSuccess) e = stream_head(s.zfrag, true, (const bf16*)B, M, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, nullptr, st);
     }
+    if (e != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
     return SLIMSPEC_OK;
 }

@@ -1,20 +1,17 @@
-// Streaming path for small M (up to 16 rows per launch): the K x V weight matrix is read from HBM
-// exactly once, in split-V slabs (one CTA per SM), every warp instruction fetching 512 contiguous
-// bytes of one row.  The logits never leave the SM: every CTA keeps max / sum-exp / top-k per
-// row for its slab, and the last CTA to finish merges the per-slab records (Section 4.1
+// Streaming path for three to sixteen rows per launch (one and two rows: stream_fma.cu): the K x V
+// weight matrix is read from HBM exactly once, in split-V slabs, every warp instruction fetching
+// 512 contiguous bytes of one row.  The logits never leave the SM: every CTA keeps max / sum-exp /
+// top-k per row for its slab, and the slab records are merged at the end (Section 4.1
 // up-projection, the softmax of Section 3.2 in online form, and the candidate selection).
 //
-// Two main loops feed one epilogue:
-//   k_stream_head_fma  one or two rows: loads held in flight in registers, packed FP32 FMAs
-//                      against the fp32 code;
-//   k_stream_head_mma  three to sixteen rows: a cp.async ring in shared memory, ldmatrix and
-//                      warp-level tensor-core instructions (mma.sync m16n8k16, bf16 in, fp32
-//                      accumulate) with the rows of the batch on the instruction's 16-row side and
-//                      the code as bf16 value + bf16 remainder.  (On this GPU one such instruction
-//                      holds the SM's legacy tensor pipe for 8 cycles: 8 of them per 2 KB of
-//                      weights keep up with HBM, 16 do not -- hence the packed fragments below.)
-// The code itself comes from k_stream_code: the same fragment scheme applied to h A, split over
-// K across the CTAs of a cluster and folded through distributed shared memory.
+//   k_stream_code      the down-projection: h A with the rows of the batch on the 16-row side of
+//                      warp-level tensor-core instructions, split over K across the CTAs of a
+//                      cluster and folded through distributed shared memory; leaves the code as
+//                      bf16 value + bf16 remainder in the form the head kernel reads.
+//   k_stream_head_mma  a cp.async ring in shared memory, ldmatrix and mma.sync m16n8k16 (bf16 in,
+//                      fp32 accumulate).  On this GPU one such instruction holds the SM's legacy
+//                      tensor pipe for 8 cycles: 8 of them per 2 KB of weights keep up with HBM,
+//                      16 do not -- hence the packed fragments below.
 #include "kernels.h"
 #include "ptx.cuh"
 #include "select.cuh"
@@ -23,23 +20,18 @@
 
 namespace slimspec {
 
-static constexpr int kHeadWarps = 14;                 // warps of a CTA of the FMA kernel (one CTA per SM)
-static constexpr int kHeadThreads = kHeadWarps * 32;
 static constexpr int kMmaWarps = 7;                   // warps of a CTA of the tensor-core kernel (two CTAs per SM): 64 columns each
 static constexpr int kMmaThreads = kMmaWarps * 32;
-static constexpr size_t kMmaSmem = 80 * 1024;         // its shared memory: two such CTAs and the down-projection's CTA of the next call share an SM
+static constexpr size_t kMmaSmem = 76 * 1024;         // its shared memory: two such CTAs and the down-projection's CTA of the next call share an SM
 static constexpr int kMaxStages = 8;                  // most stages of the shared-memory ring
 static constexpr int kCand = 256;                     // candidates one row may park in a CTA's epilogue
-enum : int { kCodeF32 = 0, kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3, kCodeRows = 4 };
+enum : int { kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3, kCodeRows = 4 };
 static constexpr size_t kZOneChunkBytes = 16 * 1024;  // code fragments up to this size stay whole in shared memory
 static constexpr size_t kZChunkBytes = 8 * 1024;      // else they pass through two buffers of this size
 static constexpr int kEpFixedBytes = 64 + (16 * 64 + 16 + 16 + 16 + 16 * 16) * 4;
-static constexpr int kFmaLoads = 16;                  // 16-byte loads a thread of the FMA kernel keeps in flight
-static constexpr size_t kFmaCodeBytes = 64 * 1024;    // most shared memory the FMA kernel spends on the code
-static constexpr size_t kFmaSmem = 158 * 1024;        // its shared memory in all: the down-projection's CTA of the next call must fit beside it
 
 struct HeadParams {
-    const uint32_t* zfrag;    // code: fragments [nkb][ZP][32 lanes][4 words], or fp32 [K][2] for the FMA kernel
+    const uint32_t* zfrag;    // code fragments [nkb][ZP][32 lanes][4 words]
     const bf16* B;            // [K][V]
     int M, K, V, k, mode;
     int ncta;                 // slabs
@@ -49,8 +41,6 @@ struct HeadParams {
     int nkb;                  // 16-row blocks of the matrix: ceil(K / 16)
     int kb_chunk, nchunks;    // blocks of code fragments per shared-memory chunk, chunks
     unsigned int zarea_bytes; // shared memory the code takes
-    int ct, rg;               // FMA kernel: column threads (one per unit of the widest slab) and row groups
-    int srows;                // FMA kernel: rows of the slab fetched into shared memory ahead of the code
     int rec_words;            // words per record: max, sum-exp, k (key, id) pairs, padded to 4
     int32_t* ids;
     float* logprobs;
@@ -64,32 +54,6 @@ struct HeadParams {
 
 // ------------------------------------------------------------------------------------------
 // Small PTX helpers of this file.
-
-// Streaming load of weights: not kept in the L1, and first in line for eviction from the L2, so
-// that the stream does not push out what is meant to stay there (the rows of the next call's
-// matrices asked for ahead of time, the down-projection matrix, the code).
-__device__ __forceinline__ uint64_t policy_evict_first()
-{
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ uint4 ldg_stream(const void* p, uint64_t pol)
-{
-    uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p), "l"(pol));
-    return r;
-}
-__device__ __forceinline__ void prefetch_l2_keep(const void* p) { asm volatile("prefetch.global.L2::evict_last [%0];" ::"l"(p)); }
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t r;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
-    return r;
-}
 
 // D (16 x 8, fp32) += A (16 x 16, bf16, row-major fragment) * B (16 x 8, bf16, column fragment)
 __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint4& a, uint32_t b0, uint32_t b1)
@@ -137,8 +101,7 @@ __device__ __forceinline__ unsigned int ticket_take(unsigned int* ticket)
     return old;
 }
 
-// The code z (or, for the full-rank head, h itself) reaches the head kernels in one of four forms:
-//   kCodeF32     fp32 [K][2]: entry (j, m) is z[m][j] (row 1 zero when M = 1): the FMA kernel
+// The code z (or, for the full-rank head, h itself) leaves this file's kernels in one of four forms:
 //   kCodePacked  fragments, one part: rows 0-7 hold the value rounded to bf16 and rows 8-15 the
 //                rounding remainders of those same rows, so ONE instruction multiplies both
 //                (M <= 8; the two halves of its result are summed at the end)
@@ -167,20 +130,25 @@ struct CodeParams {
     int M, d, r;
     int S;            // K splits = CTAs per cluster
     int nkb;          // 16-row blocks of A: ceil(d / 16)
-    int fmt;          // kCodeF32, kCodePacked, kCodeSplit or kCodeRows
+    int chunk_kbs;    // 16-row blocks of A per shared-memory buffer
+    int nbuf;         // buffers
+    int fmt;          // kCodePacked, kCodeSplit or kCodeRows
     uint32_t* zfrag;  // the code in that form
     bf16* zrows;      // kCodeRows: value [M][r]
     bf16* zrows_lo;   // kCodeRows: remainder [M][r], or null
 };
 
 static constexpr int kCodePitch = 80;            // bytes between two rows of the A slice in shared memory: 5 units (odd)
-static constexpr int kCodeChunkRows = 1024;      // rows of A a CTA holds at a time
+static constexpr int kCodeSliceRows = 640;       // rows of A a CTA holds at once when its whole share fits (50 KB: it then
+                                                 // shares the SM with a head CTA) ...
+static constexpr int kCodeChunkRows = 320;       // ... else it works through its share in chunks of this many rows,
+static constexpr int kCodeRing = 4;              // through a ring of this many buffers, two CTAs per SM
 
 __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
 {
     __shared__ __align__(16) float wt[4][16 * 32];      // the warps' partial tiles
     __shared__ __align__(16) float ct[8][16 * 32];      // the cluster's partial tiles (used in its first CTA)
-    extern __shared__ __align__(128) unsigned char aslice[];     // [rows][kCodePitch]: 32 columns of A
+    extern __shared__ __align__(128) unsigned char aslice[];     // [buffers][rows][kCodePitch]: 32 columns of A
     pdl_launch_dependents();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int rank = blockIdx.x;
@@ -189,22 +157,29 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
     const int m0 = blockIdx.z * 16;                      // first row of this CTA's tile of the batch
     const int mrows = min(16, p.M - m0);
     const bf16* hrows = p.h + (size_t)m0 * d;
-    // this CTA's run of 16-row blocks, in chunks that fit the shared memory
+    // this CTA's run of 16-row blocks, whole or in chunks through two buffers
     const int cta_kb0 = (int)((long long)p.nkb * rank / p.S), cta_kb1 = (int)((long long)p.nkb * (rank + 1) / p.S);
-    auto fetch = [&](int kb0, int kb1) {
+    const int chunk_kbs = p.chunk_kbs;
+    const int nchunks = (cta_kb1 - cta_kb0 + chunk_kbs - 1) / chunk_kbs;
+    const uint32_t buf_bytes = (uint32_t)chunk_kbs * 16u * kCodePitch;
+    const int nbuf = p.nbuf, depth = max(1, nbuf - 1);         // chunks in flight
+    auto fetch = [&](int c) {
         // weights may be read before the kernel ahead in the stream has finished: they are final before
         // the call is made (the contract of the library); only h comes from that kernel
-        const int rows = 16 * (kb1 - kb0);
-        for (int idx = tid; idx < rows * 4; idx += 128) {
-            const int row = idx >> 2, u = idx & 3;
-            const int grow = min(16 * kb0 + row, d - 1);             // rows past d re-read the last row (their h is zero)
-            const int col = min(j0 + 8 * u, r - 8);                  // a ragged last tile re-reads the last columns
-            cp_async16(aslice + (size_t)row * kCodePitch + u * 16, p.A + (size_t)grow * r + col);
+        if (c < nchunks) {
+            const int kb0 = cta_kb0 + c * chunk_kbs, kb1 = min(cta_kb1, kb0 + chunk_kbs);
+            unsigned char* dst = aslice + (size_t)(c % nbuf) * buf_bytes;
+            const int rows = 16 * (kb1 - kb0);
+            for (int idx = tid; idx < rows * 4; idx += 128) {
+                const int row = idx >> 2, u = idx & 3;
+                const int grow = min(16 * kb0 + row, d - 1);             // rows past d re-read the last row (their h is zero)
+                const int col = min(j0 + 8 * u, r - 8);                  // a ragged last tile re-reads the last columns
+                cp_async16(dst + (size_t)row * kCodePitch + u * 16, p.A + (size_t)grow * r + col);
+            }
         }
         cp_async_commit();
     };
-    const int chunk_kbs = kCodeChunkRows / 16;
-    fetch(cta_kb0, min(cta_kb1, cta_kb0 + chunk_kbs));
+    for (int c = 0; c < depth; ++c) fetch(c);
     pdl_wait();
 
     float acc[4][4];
@@ -215,18 +190,19 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
     const uint32_t lane_off = (uint32_t)((lane & 7) + ((lane >> 3) & 1) * 8) * kCodePitch + (uint32_t)(lane >> 4) * 16u;
     const uint32_t as_s = smem_u32(aslice);
 
-    for (int c0 = cta_kb0; c0 < cta_kb1; c0 += chunk_kbs) {
-        const int c1 = min(cta_kb1, c0 + chunk_kbs);
-        if (c0 > cta_kb0) { __syncthreads(); fetch(c0, c1); }
+    for (int c = 0; c < nchunks; ++c) {
+        const int c0 = cta_kb0 + c * chunk_kbs, c1 = min(cta_kb1, c0 + chunk_kbs);
         // the warp's blocks of this chunk; their h fragments are the only loads that wait for the kernel ahead
         const int n = c1 - c0;
         const int wb0 = c0 + n * warp / 4, wb1 = c0 + n * (warp + 1) / 4;
-        cp_async_wait_pending(0);
-        __syncthreads();
-        for (int kb = wb0; kb < wb1; kb += 8) {
-            uint4 hf[8];
+        cp_async_wait_pending(depth - 1);          // chunk c is in (later ones may still be on their way)
+        __syncthreads();                           // ... for everyone, and everyone is done with chunk c - 1
+        fetch(c + depth);                          // into the buffer chunk c - 1 has left
+        const uint32_t cbase = as_s + (uint32_t)(c % nbuf) * buf_bytes;
+        for (int kb = wb0; kb < wb1; kb += 4) {
+            uint4 hf[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < 4; ++i) {
                 const int k0 = 16 * (kb + i) + 2 * t;
                 const bool on = kb + i < wb1;
                 const bool lo_ok = on && k0 < d, hi_ok = on && k0 + 8 < d;
@@ -238,9 +214,9 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
                 hf[i].w = (g + 8 < mrows && hi_ok) ? __ldcg(h1 + 4) : 0u;
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < 4; ++i) {
                 if (kb + i < wb1) {
-                    const uint32_t a = as_s + (uint32_t)(kb + i - c0) * 16u * kCodePitch + lane_off;
+                    const uint32_t a = cbase + (uint32_t)(kb + i - c0) * 16u * kCodePitch + lane_off;
                     uint32_t b0, b1, b2, b3;
                     ldmatrix_x4_trans(b0, b1, b2, b3, a);
                     mma_bf16(acc[0], hf[i], b0, b1);
@@ -287,14 +263,6 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
     const int row = tid >> 3, j = j0 + (tid & 7) * 4;
     if (j >= r) return;
     const float z[4] = {v.x, v.y, v.z, v.w};
-    if (p.fmt == kCodeF32) {
-        float* zf = reinterpret_cast<float*>(p.zfrag);
-        if (row < 2) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) zf[(size_t)(j + e) * 2 + row] = z[e];
-        }
-        return;
-    }
     uint32_t hi[4], lo[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -328,18 +296,12 @@ __global__ void __launch_bounds__(128, 8) k_stream_code(const CodeParams p)
 }
 
 // The full-rank head has no down-projection: its "code" is h itself, exact in bf16
-// (kCodeF32 or kCodePlain).
-__global__ void k_stream_widen(const bf16* __restrict__ h, int M, int d, int nkb, int fmt, uint32_t* __restrict__ zfrag)
+// (kCodePlain).
+__global__ void k_stream_widen(const bf16* __restrict__ h, int M, int d, int nkb, uint32_t* __restrict__ zfrag)
 {
     pdl_launch_dependents();
     pdl_wait();          // launched early: the kernel before it may still read the code
     const int w = blockIdx.x * blockDim.x + threadIdx.x;
-    if (fmt == kCodeF32) {
-        if (w >= 2 * d) return;
-        const int j = w >> 1, m = w & 1;
-        reinterpret_cast<float*>(zfrag)[w] = m < M ? __bfloat162float(h[(size_t)m * d + j]) : 0.f;
-        return;
-    }
     if (w >= nkb * 128) return;
     const int kb = w >> 7, lane = (w >> 2) & 31, reg = w & 3;
     const int row = (lane >> 2) + 8 * (reg & 1);
@@ -350,9 +312,9 @@ __global__ void k_stream_widen(const bf16* __restrict__ h, int M, int d, int nkb
 }
 
 // ------------------------------------------------------------------------------------------
-// Epilogue of both head kernels.  The slab's logits lie in shared memory: logit (row, column c) is
-// the sum over g < ngroups of lg[g * gstride + row * lpitch + c] (the FMA kernel leaves one partial
-// sum per row group).  Thread i looks after columns i, i + blockDim, ...
+// Epilogue of the head kernel.  The slab's logits lie in shared memory: logit (row, column c) is
+// the sum over g < ngroups of lg[g * gstride + row * lpitch + c] (ngroups = 1 here; a kernel that
+// leaves one partial sum per row group may pass more).  Thread i looks after columns i, i + blockDim, ...
 //   (1) maxima of groups of eight threads; (2) a warp per row: the k-th largest of these maxima
 //   bounds the slab's k-th largest logit from below; (3) sum of exp against the slab's maximum,
 //   logits that reach the bound are parked; (4) a warp per row orders the parked candidates by
@@ -529,135 +491,6 @@ __device__ __forceinline__ void slab_epilogue(const HeadParams& p, unsigned char
 }
 
 // ------------------------------------------------------------------------------------------
-// One or two rows.  One CTA per V slab; thread = (column unit of 8 columns, row group).  Every
-// thread keeps 16 loads of its unit in flight (rows g, g + RG, g + 2 RG, ...) in two alternating
-// register sets, so that a wait for the older set never waits for loads issued after it,
-// multiplies each arriving row by the code held in shared memory as (z, z) pairs (packed FP32
-// FMAs) and refills.  The row groups' partial sums meet in shared memory.
-// While the code is not there yet (the kernel comes up early, under the tail of the call before),
-// HBM would idle: the first `srows` rows of the slab are fetched into shared memory (cp.async) and
-// the next 16 per thread into the registers, all before the wait; the main loop then works these
-// off together with what it streams.  (Asking the L2 for rows ahead of time instead was measured
-// and gains nothing: an L2 hit is served little faster than HBM serves a miss.)
-// The weights may be read before the preceding kernel has finished because they are final before
-// the call is made (the contract of the library); only the code depends on that kernel.
-template <int MT>
-__global__ void __launch_bounds__(512, 1) k_stream_head_fma(const HeadParams p)
-{
-    extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char* zarea = smem + ((kEpFixedBytes + 127) / 128) * 128;
-    float2* zs = reinterpret_cast<float2*>(zarea);              // [K][MT] (z, z) pairs
-    unsigned char* pre = zarea + p.zarea_bytes;                 // [srows][CT * 16]: the slab's first rows; later the partial sums
-    float* red = reinterpret_cast<float*>(pre);                 // [RG][MT][lpitch] partial sums, then the epilogue's lists
-    const int tid = threadIdx.x;
-    const int CT = p.ct, RG = p.rg, S = p.srows;
-    const int g = tid / CT, c = tid - g * CT;                   // row group, column unit
-    const int cta = blockIdx.x;
-    const int K = p.K;
-    const size_t Vb = (size_t)p.V * sizeof(bf16);
-    const int my_units = p.units_base + (cta < p.units_rem ? 1 : 0);
-    const int unit0 = cta * p.units_base + min(cta, p.units_rem);
-    const char* slab = reinterpret_cast<const char*>(p.B + (size_t)unit0 * 8);
-    const int lpitch = CT * 8;
-    const uint32_t prow = (uint32_t)CT * 16u;                   // bytes between two preloaded rows
-
-    constexpr int U = kFmaLoads, UH = U / 2;
-    const bool active = g < RG && c < my_units;
-    const char* base = slab + (size_t)c * 16 + (size_t)S * Vb;  // the register pipeline starts behind the preloaded rows
-    const int KR = K - S;                                       // rows it covers
-    const int stepU = RG * U;
-    const uint64_t pol = policy_evict_first();
-    uint4 q[2][UH];
-    if (active) {
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-            for (int j = 0; j < UH; ++j) {
-                const int row = g + (hh * UH + j) * RG;
-                q[hh][j] = row < KR ? ldg_stream(base + (size_t)row * Vb, pol) : make_uint4(0u, 0u, 0u, 0u);
-            }
-    }
-    for (int idx = tid; idx < S * my_units; idx += blockDim.x) {
-        const int row = idx / my_units, cc = idx - row * my_units;
-        cp_async16(pre + (size_t)row * prow + (size_t)cc * 16, slab + (size_t)row * Vb + (size_t)cc * 16);
-    }
-    cp_async_commit();
-    pdl_launch_dependents();
-    if (p.wait_prev) pdl_wait();
-    for (int i = tid; i < 16 * 64; i += blockDim.x) reinterpret_cast<float*>(smem + 64)[i] = -FLT_MAX;
-    // the code: fp32 [K][2] in global memory -> (z, z) pairs
-    {
-        const float* zf = reinterpret_cast<const float*>(p.zfrag);
-        for (int e = tid; e < K * MT; e += blockDim.x) {
-            const int j = e / MT, m = e - j * MT;
-            const float zv = __ldcg(zf + (size_t)j * 2 + m);
-            zs[e] = make_float2(zv, zv);
-        }
-    }
-    cp_async_wait_pending(0);
-    __syncthreads();
-
-    float2 acc[MT][4];
-#pragma unroll
-    for (int m = 0; m < MT; ++m)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) acc[m][e] = make_float2(0.f, 0.f);
-    auto fma_row = [&](const uint4& w4, int zrow) {
-        const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-        float2 b2[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) b2[e] = make_float2(__uint_as_float(w[e] << 16), __uint_as_float(w[e] & 0xffff0000u));
-        const float2* zr = zs + (size_t)zrow * MT;
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            const float2 z2 = zr[m];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[m][e] = __ffma2_rn(b2[e], z2, acc[m][e]);
-        }
-    };
-    if (active) {
-        // preloaded rows of this thread: g, g + RG, ... below S, a few per block of streamed rows
-        int srow = g;
-        const int nblocks = (KR + stepU - 1) / stepU;
-        const int mine = (S - g + RG - 1) / RG;
-        const int per_block = nblocks > 0 ? (mine + nblocks - 1) / nblocks : mine;
-        const unsigned char* pcol = pre + (size_t)c * 16;
-        for (int row = g; row < KR; row += stepU) {
-            const bool checked = row - g + 2 * stepU > KR;       // this block or its refills reach past the end
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-#pragma unroll
-                for (int j = 0; j < UH; ++j) {
-                    const int rj = row + (hh * UH + j) * RG;
-                    if (!checked || rj < KR) fma_row(q[hh][j], S + rj);
-                }
-                // the set is used up: refill all of it at once
-#pragma unroll
-                for (int j = 0; j < UH; ++j) {
-                    const int nr = row + (hh * UH + j) * RG + stepU;
-                    if (!checked || nr < KR) q[hh][j] = ldg_stream(base + (size_t)nr * Vb, pol);
-                }
-            }
-            for (int i = 0; i < per_block && srow < S; ++i, srow += RG)
-                fma_row(*reinterpret_cast<const uint4*>(pcol + (size_t)srow * prow), srow);
-        }
-        for (; srow < S; srow += RG) fma_row(*reinterpret_cast<const uint4*>(pcol + (size_t)srow * prow), srow);
-    }
-    __syncthreads();            // every thread is done with the preloaded rows: their memory takes the partial sums
-    if (g < RG && c < CT) {
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            float* dst = red + ((size_t)g * MT + m) * lpitch + c * 8;
-            *reinterpret_cast<float4*>(dst) = make_float4(acc[m][0].x, acc[m][0].y, acc[m][1].x, acc[m][1].y);
-            *reinterpret_cast<float4*>(dst + 4) = make_float4(acc[m][2].x, acc[m][2].y, acc[m][3].x, acc[m][3].y);
-        }
-    }
-    __syncthreads();
-    unsigned char* lists = reinterpret_cast<unsigned char*>(red + (size_t)RG * MT * lpitch);
-    slab_epilogue<MT>(p, smem, lists, zarea, red, RG, MT * lpitch, lpitch, my_units * 8, unit0 * 8);
-}
-
-// ------------------------------------------------------------------------------------------
 // Three to sixteen rows.  One CTA per V slab, seven warps, two CTAs per SM: all warps of a CTA meet
 // at a barrier once per stage and then issue their tensor-core instructions together, so a second,
 // independent CTA on the SM keeps the tensor pipe and the memory system busy meanwhile (one CTA of
@@ -825,10 +658,8 @@ __global__ void __launch_bounds__(256, 2) k_stream_head_mma(const HeadParams p) 
 
 // ------------------------------------------------------------------------------------------
 struct Geometry {
-    int fma;             // 1: the FMA kernel (M <= 2), 0: the tensor-core kernel
     int ncta, units_base, units_rem, rec_words;
-    int ct, rg, srows;                                       // FMA kernel
-    int nch, pitch_units, ns, nkb, kb_chunk, nchunks;        // tensor-core kernel
+    int nch, pitch_units, ns, nkb, kb_chunk, nchunks;
     size_t zarea_bytes, smem;
 };
 
@@ -837,45 +668,15 @@ static constexpr size_t kHeadSmemMax = 226 * 1024;
 static size_t merge_bytes(int) { return (size_t)(16 + 2 * 16 * 32 + 16 * 2 * kMergeCand) * 4; }
 
 // zparts: 1 or 2 parts of code fragments (tensor-core kernel)
-static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, bool want_fma, Geometry* g)
+static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, Geometry* g)
 {
     if (V % 8 != 0 || K < 1 || k > 32 || k < 1 || M < 1 || M > 16) return false;
     const int units = V / 8;
-    int ncta = sm_count;
-    if (ncta > units) ncta = units;
-    if (ncta > kMaxRecords) ncta = kMaxRecords;
-    g->ncta = ncta;
-    g->units_base = units / ncta;
-    g->units_rem = units % ncta;
-    const int max_units = g->units_base + (g->units_rem ? 1 : 0);
     g->rec_words = (2 + 2 * k + 3) / 4 * 4;
     const size_t fixed0 = ((kEpFixedBytes + 127) / 128) * 128;
-    g->fma = 0;
-    if (want_fma && M <= 2 && max_units <= kHeadThreads) {
-        const int mt = M;
-        g->ct = max_units;
-        int rg = kHeadThreads / g->ct;
-        if (rg > 16) rg = 16;
-        if (rg > K) rg = K;
-        g->rg = rg;
-        g->zarea_bytes = ((size_t)K * mt * 8 + 127) / 128 * 128;
-        const size_t red = (size_t)rg * mt * g->ct * 8 * 4;
-        const size_t cand = (size_t)mt * kCand * 8;
-        size_t rest = red + cand;
-        if (g->zarea_bytes + rest < merge_bytes(ncta)) rest = merge_bytes(ncta) - g->zarea_bytes;
-        // what is left up to kFmaSmem holds the slab's first rows (the area is reused afterwards)
-        const size_t used = fixed0 + g->zarea_bytes;
-        const size_t prow = (size_t)g->ct * 16;
-        int srows = used + rest < kFmaSmem ? (int)((kFmaSmem - used) / prow) : (int)(rest / prow);
-        if (srows > K) srows = K;
-        g->srows = srows;
-        if ((size_t)srows * prow > rest) rest = (size_t)srows * prow;
-        g->smem = used + rest;
-        if (g->zarea_bytes <= kFmaCodeBytes && g->smem <= kHeadSmemMax) { g->fma = 1; return true; }
-    }
     const int mt = M <= 8 ? 8 : 16;
-    // the tensor-core kernel: two CTAs per SM
-    ncta = 2 * sm_count;
+    // two CTAs per SM
+    int ncta = 2 * sm_count;
     if (ncta > units) ncta = units;
     if (ncta > kMaxRecords) ncta = kMaxRecords;
     g->ncta = ncta;
@@ -915,7 +716,7 @@ static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, bool 
 // The form of the code the head kernel for (M, low-rank or not) reads.
 static int code_format(const Geometry& g, int M, bool lowrank)
 {
-    if (g.fma) return kCodeF32;
+    (void)g;
     if (!lowrank) return kCodePlain;
     return M <= 8 ? kCodePacked : kCodeSplit;
 }
@@ -925,7 +726,7 @@ StreamPlan stream_plan(int M, int K, int V, int k, int sm_count)
     StreamPlan sp = {0, 0, 0, 0, 0};
     if (M < 1) return sp;
     Geometry g;
-    if (!geometry(M > 16 ? 16 : M, 2, K, V, k, sm_count, true, &g)) return sp;
+    if (!geometry(M > 16 ? 16 : M, 2, K, V, k, sm_count, &g)) return sp;
     sp.ok = 1;
     sp.mt = M <= 8 ? 8 : 16;
     sp.ncta = g.ncta;
@@ -939,7 +740,7 @@ size_t stream_code_bytes(int K) { return (size_t)((K + 15) / 16) * 2 * 512 + 102
 static bool plan_code(int M, bool lowrank, int K, int V, int k, int sm_count, Geometry* g, int* fmt)
 {
     const int zparts = (lowrank && M > 8) ? 2 : 1;
-    if (!geometry(M, zparts, K, V, k, sm_count, true, g)) return false;
+    if (!geometry(M, zparts, K, V, k, sm_count, g)) return false;
     *fmt = code_format(*g, M, lowrank);
     return true;
 }
@@ -953,16 +754,22 @@ static cudaError_t launch_code(CodeParams cp, int sm_count, cudaStream_t st)
     cp.nkb = (cp.d + 15) / 16;
     const int nct = (cp.r + 31) / 32;
     const int ntiles = (cp.M + 15) / 16;
+    // One CTA per SM at most while a CTA's whole share of A fits beside a head CTA; a larger A goes
+    // through a ring of buffers with two CTAs per SM (what counts then is the bandwidth of this kernel).
     int S = 8;
-    while (S > 1 && (S * nct > 2 * sm_count || S * 4 > cp.nkb)) S >>= 1;
+    while (S > 1 && (S * nct * ntiles > sm_count || S * 4 > cp.nkb)) S >>= 1;
+    if (((cp.nkb + S - 1) / S) * 16 > kCodeSliceRows) {
+        S = 8;
+        while (S > 1 && (S * nct * ntiles > 2 * sm_count || S * 4 > cp.nkb)) S >>= 1;
+    }
     cp.S = S;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(S, nct, ntiles);
     cfg.blockDim = dim3(128);
     {
         const int kbs = (cp.nkb + S - 1) / S;
-        const int rows = 16 * (kbs < kCodeChunkRows / 16 ? kbs : kCodeChunkRows / 16);
-        cfg.dynamicSmemBytes = (size_t)rows * kCodePitch + 128;
+        if (kbs * 16 <= kCodeSliceRows) { cp.chunk_kbs = kbs; cp.nbuf = 1; cfg.dynamicSmemBytes = (size_t)kbs * 16 * kCodePitch + 128; }
+        else { cp.chunk_kbs = kCodeChunkRows / 16; cp.nbuf = kCodeRing; cfg.dynamicSmemBytes = (size_t)kCodeRing * kCodeChunkRows * kCodePitch + 128; }
     }
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -1004,7 +811,7 @@ cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* zf
     int fmt;
     if (!plan_code(M, false, d, V, k, sm_count, &g, &fmt)) return cudaErrorInvalidValue;
     const int nkb = (d + 15) / 16;
-    const int n = fmt == kCodeF32 ? 2 * d : nkb * 128;
+    const int n = nkb * 128;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((n + 255) / 256);
     cfg.blockDim = dim3(256);
@@ -1014,7 +821,7 @@ cudaError_t stream_widen(const bf16* h, int M, int d, int V, int k, uint32_t* zf
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, k_stream_widen, h, M, d, nkb, fmt, zfrag);
+    return cudaLaunchKernelEx(&cfg, k_stream_widen, h, M, d, nkb, zfrag);
 }
 
 // Once per device: load the kernels of this file and allow the head kernels their dynamic shared
@@ -1030,10 +837,8 @@ cudaError_t stream_prepare()
     cudaError_t e;
     cudaFuncAttributes fa;
     if ((e = cudaFuncGetAttributes(&fa, k_stream_code)) != cudaSuccess) return e;
-    if ((e = cudaFuncSetAttribute(k_stream_code, cudaFuncAttributeMaxDynamicSharedMemorySize, kCodeChunkRows * kCodePitch + 128)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(k_stream_code, cudaFuncAttributeMaxDynamicSharedMemorySize, kCodeRing * kCodeChunkRows * kCodePitch + 128)) != cudaSuccess) return e;
     if ((e = cudaFuncGetAttributes(&fa, k_stream_widen)) != cudaSuccess) return e;
-    if ((e = allow_smem(k_stream_head_fma<1>)) != cudaSuccess) return e;
-    if ((e = allow_smem(k_stream_head_fma<2>)) != cudaSuccess) return e;
     if ((e = allow_smem(k_stream_head_mma<8, 1, 1>)) != cudaSuccess) return e;
     if ((e = allow_smem(k_stream_head_mma<8, 1, 2>)) != cudaSuccess) return e;
     if ((e = allow_smem(k_stream_head_mma<16, 1, 1>)) != cudaSuccess) return e;
@@ -1048,7 +853,7 @@ static cudaError_t launch_head(Kern kern, const HeadParams& hp, const Geometry& 
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(hp.ncta);
-    cfg.blockDim = dim3(g.fma ? kHeadThreads : kMmaThreads);
+    cfg.blockDim = dim3(kMmaThreads);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -1079,10 +884,7 @@ cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int 
     hp.merge_inside = (mode == 1 || M <= 7) ? 1 : 0;       // measured: from 8 rows on the merge kernel is faster (2 us at 8 rows)
     const bool pdl = after_producer_kernel;
     cudaError_t e;
-    if (g.fma) {
-        hp.ct = g.ct; hp.rg = g.rg; hp.srows = g.srows;
-        e = M == 1 ? launch_head(k_stream_head_fma<1>, hp, g, pdl, st) : launch_head(k_stream_head_fma<2>, hp, g, pdl, st);
-    } else {
+    {
         hp.pitch_units = g.pitch_units; hp.ns = g.ns;
         hp.nkb = g.nkb; hp.kb_chunk = g.kb_chunk; hp.nchunks = g.nchunks;
         if (fmt == kCodeSplit)
