@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture on this workload, see profiles/stream_head_fma_c1_m1.md), keyed by the SHA-256 of the kernel's source
+# capture on this workload, see profiles/fma_head_c1_m1.md), keyed by the SHA-256 of the kernel's source
 # file at the time of the capture: a changed source reports null.
 KNOWN_TRAFFIC = {
 }
@@ -46,7 +46,7 @@ KNOWN_TRAFFIC = {
 
 def kernel_traffic():
     import hashlib
-    path = os.path.join(ROOT, "paper_2605_10453_b200", "csrc", "stream.cu")
+    path = os.path.join(ROOT, "paper_2605_10453_b200", "csrc", "stream_fma.cu")
     try:
         with open(path, "rb") as f:
             return KNOWN_TRAFFIC.get(hashlib.sha256(f.read()).hexdigest())
@@ -377,7 +377,7 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
-        "roofline": {"bound": "hbm", "kernel": "k_stream_head_fma", "achieved": achieved, "peak": peaks["hbm_gbs"],
+        "roofline": {"bound": "hbm", "kernel": "k_fma_head", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": kernel_traffic(),
                      "peak_kind": "of " + peaks_kind, "bytes_per_launch": kern_bytes, "us_per_launch": kern_us,
                      "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,

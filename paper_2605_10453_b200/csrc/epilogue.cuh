@@ -1,0 +1,204 @@
+// Epilogue shared by the streaming head kernels: from a slab's logits in shared memory to the
+// slab's record (maximum, sum of exp, the k best (key, id) pairs), and the merge of all records by
+// the last CTA to arrive (softmax of Section 3.2 in online form, and the candidate selection).
+#pragma once
+#include "ptx.cuh"
+#include "select.cuh"
+#include <float.h>
+
+namespace slimspec {
+
+static constexpr int kCand = 256;                     // candidates one row may park in a CTA's epilogue
+// shared memory the epilogue keeps at the start of the CTA's dynamic area: ticket, group maxima
+// [16][64], bound / maximum / count per row, sums of exp [16][16]
+static constexpr int kEpFixedBytes = 64 + (16 * 64 + 16 + 16 + 16 + 16 * 16) * 4;
+
+// Arrival counter with release / acquire semantics at GPU scope: what the CTA wrote before its
+// barrier is visible to whoever reads the counter's later values.
+__device__ __forceinline__ unsigned int ticket_take(unsigned int* ticket)
+{
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(ticket) : "memory");
+    return old;
+}
+
+// ------------------------------------------------------------------------------------------
+// Epilogue of the head kernel.  The slab's logits lie in shared memory: logit (row, column c) is
+// the sum over g < ngroups of lg[g * gstride + row * lpitch + c] (ngroups = 1 here; a kernel that
+// leaves one partial sum per row group may pass more).  Thread i looks after columns i, i + blockDim, ...
+//   (1) maxima of groups of eight threads; (2) a warp per row: the k-th largest of these maxima
+//   bounds the slab's k-th largest logit from below; (3) sum of exp against the slab's maximum,
+//   logits that reach the bound are parked; (4) a warp per row orders the parked candidates by
+//   counting and writes the slab's record; then the arrival ticket, and the last CTA merges the
+//   records of every row the same way.
+// Nothing here depends on the order in which threads or CTAs arrive: results are reproducible.
+template <int MT, class Params>
+__device__ __forceinline__ void slab_epilogue(const Params& p, unsigned char* smem, unsigned char* scratch, unsigned char* merge_area,
+                                              const float* lg, int ngroups, int gstride, int lpitch, int ncols, int col_base)
+{
+    unsigned int* s_ticket = reinterpret_cast<unsigned int*>(smem);
+    float* gmax_s = reinterpret_cast<float*>(smem + 64);      // [16 rows][64]: maxima of thread groups
+    float* tau_s = gmax_s + 16 * 64;                          // [16] candidates must reach this
+    float* cmax_s = tau_s + 16;                               // [16] the slab's maximum
+    int* cnt_s = reinterpret_cast<int*>(cmax_s + 16);         // [16] candidates parked
+    float* wsum_s = reinterpret_cast<float*>(cnt_s + 16);     // [16 rows][16 warps] sums of exp
+    uint32_t* ck = reinterpret_cast<uint32_t*>(scratch);      // [MT][kCand]
+    int* ci = reinterpret_cast<int*>(ck + MT * kCand);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nt = blockDim.x, nw = nt >> 5;
+    const int cta = blockIdx.x, k = p.k;
+    const int mrows = min(p.M, MT);
+    auto logit = [&](int row, int c) {
+        float x = lg[row * lpitch + c];
+        for (int gi = 1; gi < ngroups; ++gi) x += lg[gi * gstride + row * lpitch + c];
+        return x + 0.f;             // -0 becomes +0: keys and float compares then agree
+    };
+
+    if (p.mode == 1) {
+        for (int row = 0; row < mrows; ++row)
+            for (int c = tid; c < ncols; c += nt) p.logits[(size_t)row * p.V + col_base + c] = logit(row, c);
+        return;
+    }
+    // ---- (1)  (rows in batches, so that their shuffle chains overlap)
+    constexpr int RB = MT < 4 ? MT : 4;
+    for (int row0 = 0; row0 < mrows; row0 += RB) {
+        float m[RB];
+#pragma unroll
+        for (int i = 0; i < RB; ++i) m[i] = -FLT_MAX;
+        for (int c = tid; c < ncols; c += nt) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i)
+                if (row0 + i < mrows) m[i] = fmaxf(m[i], logit(row0 + i, c));
+        }
+#pragma unroll
+        for (int o = 1; o <= 4; o <<= 1) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], o));
+        }
+        if ((lane & 7) == 0) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i)
+                if (row0 + i < mrows) gmax_s[(row0 + i) * 64 + warp * 4 + (lane >> 3)] = m[i];
+        }
+    }
+    __syncthreads();
+    // ---- (2)  Up to 16 candidates wanted, the maxima of slot pairs do (32 values, half the
+    // shuffles); beyond that all 64 slots are ranked.  (Kept as one short loop: a version that ran the
+    // rounds of a warp's rows interleaved grew the kernels by 40 % and cost 2.5 us per call.)
+    for (int row = warp; row < mrows; row += nw) {
+        const uint32_t ka = f2key(gmax_s[row * 64 + lane]), kb2 = f2key(gmax_s[row * 64 + 32 + lane]);
+        const uint32_t kth = (k <= 16) ? warp_kth_largest_any(max(ka, kb2), k, lane) : warp_kth_largest64(ka, kb2, min(k, 64), lane);
+        const uint32_t mx = warp_max_u32(max(ka, kb2));
+        if (lane == 0) { tau_s[row] = key2f(kth); cmax_s[row] = key2f(mx); cnt_s[row] = 0; }
+    }
+    __syncthreads();
+    // ---- (3)
+    for (int row0 = 0; row0 < mrows; row0 += RB) {
+        float s[RB], tau[RB], cm[RB];
+#pragma unroll
+        for (int i = 0; i < RB; ++i) {
+            const int row = min(row0 + i, mrows - 1);
+            s[i] = 0.f; tau[i] = tau_s[row]; cm[i] = cmax_s[row];
+        }
+        for (int c = tid; c < ncols; c += nt) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i) {
+                if (row0 + i < mrows) {
+                    const int row = row0 + i;
+                    const float x = logit(row, c);
+                    s[i] += __expf(x - cm[i]);
+                    if (x >= tau[i]) {
+                        const int pos = atomicAdd(&cnt_s[row], 1);
+                        if (pos < kCand) { ck[row * kCand + pos] = f2key(x); ci[row * kCand + pos] = col_base + c; }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i) s[i] += __shfl_xor_sync(0xffffffffu, s[i], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int i = 0; i < RB; ++i)
+                if (row0 + i < mrows) wsum_s[(row0 + i) * 16 + warp] = s[i];
+        }
+    }
+    __syncthreads();
+    // ---- (4)
+    const int P = p.ncta;
+    const int RW = p.rec_words;
+    for (int row = warp; row < mrows; row += nw) {
+        float* rec = p.part + ((size_t)row * P + cta) * RW;
+        {
+            const float s = warp_sum(lane < nw ? wsum_s[row * 16 + lane] : 0.f);      // fixed order: reproducible
+            if (lane == 0) *reinterpret_cast<float2*>(rec) = make_float2(cmax_s[row], s);
+        }
+        const int n = cnt_s[row];
+        if (n <= kCand) {
+            // the (key, id) pairs go straight into the record: rank j to words 2 + 2 j, 3 + 2 j
+            const uint32_t* rk = ck + row * kCand;
+            const int* ri = ci + row * kCand;
+            for (int base = 0; base < n; base += 32) {
+                const int i = base + lane;
+                const uint32_t mk = i < n ? rk[i] : 0u;
+                const int mi = i < n ? ri[i] : kNoId;
+                int rank = 0;
+                for (int j = 0; j < n; ++j) rank += better(rk[j], ri[j], mk, mi) ? 1 : 0;
+                if (i < n && rank < k) *reinterpret_cast<float2*>(rec + 2 + 2 * rank) = make_float2(__uint_as_float(mk), __int_as_float(mi));
+            }
+            for (int j = n + lane; j < k; j += 32) *reinterpret_cast<float2*>(rec + 2 + 2 * j) = make_float2(__uint_as_float(0u), __int_as_float(kNoId));
+        } else {
+            // Slow path (masses of equal logits, or logits in long ordered runs): k rounds over the
+            // row, each taking the best logit that comes after the previous winner in the order;
+            // nothing is kept between rounds but that winner.
+            uint32_t lk = 0xffffffffu;
+            int li = -1;
+            for (int j = 0; j < k; ++j) {
+                uint32_t bk = 0u;
+                int bi = kNoId;
+                for (int c = lane; c < ncols; c += 32) {
+                    const uint32_t ke = f2key(logit(row, c));
+                    const int ie = col_base + c;
+                    if (after(ke, ie, lk, li) && better(ke, ie, bk, bi)) { bk = ke; bi = ie; }
+                }
+                const uint32_t wk = warp_max_u32(bk);
+                const uint32_t wi = warp_min_u32(bk == wk ? (uint32_t)bi : 0xffffffffu);
+                lk = wk;
+                li = (int)wi;
+                if (lane == 0) *reinterpret_cast<float2*>(rec + 2 + 2 * j) = make_float2(__uint_as_float(wk), __int_as_float(wk != 0u ? (int)wi : kNoId));
+                if (wk == 0u) { lk = 0u; li = kNoId; }      // nothing left: later rounds stay empty
+            }
+        }
+    }
+
+    // ---- arrival: the last CTA merges the records of every row (many rows: a kernel of its own does,
+    // with two warps per row on as many SMs as it takes)
+    if (!p.merge_inside) return;
+    __syncthreads();
+    if (tid == 0) *s_ticket = ticket_take(p.ticket);
+    __syncthreads();
+    if (*s_ticket != (unsigned)(p.ncta - 1)) return;
+
+    // Two tasks per row, a warp each: the row's log-sum-exp, and its k best entries.
+    float* lse_s = reinterpret_cast<float*>(merge_area);                 // [16]
+    uint32_t* ok_all = reinterpret_cast<uint32_t*>(lse_s + 16);          // [16 rows][32] ordered keys
+    int* oi_all = reinterpret_cast<int*>(ok_all + 16 * 32);              // [16 rows][32] their ids
+    uint32_t* mk = reinterpret_cast<uint32_t*>(oi_all + 16 * 32) + warp * 2 * kMergeCand;     // this warp's candidates
+    int* mi = reinterpret_cast<int*>(mk + kMergeCand);
+    for (int task = warp; task < 2 * p.M; task += nw) {
+        const int row = task >> 1;
+        if (P <= 5 * 32) merge_task<5>(p.part, P, RW, k, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+        else merge_task<kMergeLists>(p.part, P, RW, k, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+    }
+    __syncthreads();
+    for (int e = tid; e < p.M * k; e += nt) {
+        const int row = e / k, j = e - row * k;
+        p.ids[e] = oi_all[row * 32 + j];
+        p.logprobs[e] = key2f(ok_all[row * 32 + j]) - lse_s[row];
+    }
+    if (tid == 0) *p.ticket = 0;
+}
+
+}  // namespace slimspec
