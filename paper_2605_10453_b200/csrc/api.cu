@@ -14,6 +14,7 @@ struct slimspec_ctx {
     int forced_path;
     int last_path;
     long long launches;
+    unsigned int epoch;   // number of the last one- or two-row call (the code it publishes carries it)
     Scratch s;
     bf16* h_stage;        // device copy of host activations (head_topk_host)
     // Results of head_topk_host: pinned host memory mapped into the device, so the kernels write
@@ -87,6 +88,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     ok = ok && cudaMalloc(&c->s.z, z_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.part, part_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zfrag, stream_code_bytes(max_d)) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->s.zq, fma_code_words(max_d) * sizeof(uint2)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zpart, zpart_elems * sizeof(float)) == cudaSuccess;
     ok = ok && cudaMalloc(&c->s.zb, 2 * mpad128 * (size_t)max_d * sizeof(bf16)) == cudaSuccess;
     if (ok) c->s.zb_lo = c->s.zb + mpad128 * (size_t)max_d;
@@ -111,6 +113,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     }
     ok = ok && cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.err, 0, sizeof(int)) == cudaSuccess;
+    ok = ok && cudaMemset(c->s.zq, 0, fma_code_words(max_d) * sizeof(uint2)) == cudaSuccess;
     ok = ok && cudaMemset(c->s.z, 0, z_elems * sizeof(float)) == cudaSuccess;
     ok = ok && stream_prepare() == cudaSuccess && fma_prepare() == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
@@ -127,7 +130,7 @@ extern "C" void slimspec_destroy(slimspec_ctx* c)
 {
     if (!c) return;
     cudaDeviceSynchronize();
-    cudaFree(c->s.z); cudaFree(c->s.zfrag); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.smax); cudaFree(c->s.thr0); cudaFree(c->s.tickets); cudaFree(c->s.err);
+    cudaFree(c->s.z); cudaFree(c->s.zfrag); cudaFree(c->s.zq); cudaFree(c->s.part); cudaFree(c->s.zpart); cudaFree(c->s.zb); cudaFree(c->s.smax); cudaFree(c->s.thr0); cudaFree(c->s.tickets); cudaFree(c->s.err);
     cudaFree(c->s.logits); cudaFree(c->h_stage);
     if (c->res_host) cudaFreeHost(c->res_host);
     if (c->ev0) {
@@ -316,15 +319,13 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
         const bf16* hm = h + (size_t)m0 * d;
         const int kk = mode == 0 ? k : 1;
         int nl = 0;
-        // one or two rows: the FMA kernels; three to sixteen: the tensor-core streaming kernels
-        const FmaPlan fp = fma_plan(mrows, d, K, V, kk, c->sm_count);
+        // one or two rows: the FMA kernel, one launch; three to sixteen: the tensor-core streaming kernels
+        const FmaPlan fp = fma_plan(mrows, d, lowrank ? r : 0, V, kk, c->sm_count);
         const bool fma = fp.ok && fp.ncta <= c->s.max_parts;
-        if (fma) {
-            if (lowrank) CK(fma_downproj(hm, A, mrows, fp.mt, d, r, c->s, st));
-            else CK(fma_widen_t(hm, mrows, fp.mt, d, c->s.z, st));
-        } else {
+        if (!fma) {
             if (lowrank) CK(stream_code(hm, A, mrows, d, r, V, kk, c->s.zfrag, c->sm_count, st));
             else CK(stream_widen(hm, mrows, d, V, kk, c->s.zfrag, c->sm_count, st));
+            nl = 1;
         }
         int slot = -1;
         if (c->timing_on) {
@@ -332,18 +333,24 @@ static int run_head(slimspec_ctx* c, const bf16* h, const bf16* A, const bf16* B
             slot = c->timing_used++;
             CK(cudaEventRecord(c->ev0[slot], st));
         }
-        // an event between the two kernels serialises them: the timed kernel then runs alone
+        // an event between two kernels serialises them: the timed kernel then runs alone
         int32_t* ids_t = mode == 0 ? ids + (size_t)m0 * k : nullptr;
         float* lp_t = mode == 0 ? logprobs + (size_t)m0 * k : nullptr;
         float* lg_t = mode == 1 ? logits + (size_t)m0 * V : nullptr;
         if (fma) {
-            CK(fma_head(c->s.z, Bm, mrows, fp.mt, K, V, kk, mode, ids_t, lp_t, lg_t, c->s, c->sm_count, slot < 0, st));
-            nl = 1;
+            if (++c->epoch == 0) {      // the call numbers have gone round: forget the old ones
+                CK(cudaMemsetAsync(c->s.zq, 0, fma_code_words(c->max_d) * sizeof(uint2), st));
+                c->epoch = 1;
+            }
+            CK(fma_head(hm, A, Bm, mrows, fp.mt, d, r, V, kk, mode, ids_t, lp_t, lg_t, c->s, c->epoch, c->sm_count, st));
+            nl += 1;
         } else {
-            CK(stream_head(c->s.zfrag, lowrank, Bm, mrows, K, V, kk, mode, ids_t, lp_t, lg_t, c->s, c->sm_count, slot < 0, &nl, st));
+            int nh = 0;
+            CK(stream_head(c->s.zfrag, lowrank, Bm, mrows, K, V, kk, mode, ids_t, lp_t, lg_t, c->s, c->sm_count, slot < 0, &nh, st));
+            nl += nh;
         }
         if (slot >= 0) CK(cudaEventRecord(c->ev1[slot], st));
-        c->launches += 1 + nl;
+        c->launches += nl;
     }
     return SLIMSPEC_OK;
 }

@@ -13,7 +13,7 @@ typedef __nv_bfloat16 bf16;
 // slab's k best (logit, id) pairs in (logit desc, id asc) order.
 // Layout in the context's scratch: float pm[P], ps[P], pv[P][k]; int pi[P][k] per row.
 struct Scratch {
-    float* z;            // fp32 code (or widened h): generic path [M][K]; one- and two-row streaming path transposed, [K][mt]
+    float* z;            // fp32 code (or widened h): generic path [M][K]; one- and two-row streaming path: partial sums [splits][K][mt]
     uint32_t* zfrag;     // streaming path: the code, as fp32 or as tensor-core fragments (see stream.cu)
     bf16* zb;            // bf16 code [M][r] for the tensor-core path
     bf16* zb_lo;         // its rounding remainder (z - zb), bf16: used while the call is HBM-bound
@@ -25,6 +25,7 @@ struct Scratch {
     float* part;         // split-V partial records
     size_t part_elems;
     unsigned int* tickets;  // arrival counters (self-resetting)
+    uint2* zq;              // one- and two-row path: the code as published (value, call number) words; no other path writes here
     int* err;            // device error word
     float* logits;       // generic path only: M x V fp32, grown on demand
     size_t logits_elems;
@@ -40,21 +41,22 @@ cudaError_t generic_softmax_topk(const float* logits, int M, int V, int k, int32
 
 // ---- streaming path, one or two rows (stream_fma.cu) ------------------------------------
 struct FmaPlan {
-    int ok;          // 0: shapes not supported by these kernels
+    int ok;          // 0: shapes not supported by this kernel
     int mt;          // rows per launch (1 or 2)
     int ncta;        // V slabs = CTAs
     int launches;    // kernels per call
 };
-FmaPlan fma_plan(int M, int d, int K, int V, int k, int sm_count);
+// r = 0: the full-rank head (the streamed matrix has d rows).
+FmaPlan fma_plan(int M, int d, int r, int V, int k, int sm_count);
 cudaError_t fma_prepare();
-// z^T = (h A)^T for M <= 2 rows (fp32, [r][mt], rows M..mt-1 zero-filled); r must be a multiple of 16.
-cudaError_t fma_downproj(const bf16* h, const bf16* A, int M, int mt, int d, int r, const Scratch& s, cudaStream_t st);
-// z^T = widened h^T (full-rank head: no down-projection).
-cudaError_t fma_widen_t(const bf16* h, int M, int mt, int d, float* zT, cudaStream_t st);
-// logits = z B streamed once; mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.
-cudaError_t fma_head(const float* z, const bf16* B, int M, int mt, int K, int V, int k, int mode,
-                     int32_t* ids, float* logprobs, float* logits, const Scratch& s, int sm_count,
-                     bool after_producer_kernel, cudaStream_t st);
+// The whole head for M <= 2 rows in one launch: z = h A (A null: z = h), logits = z B streamed once;
+// mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.  Uses s.zq
+// (fma_code_words(max r) 8-byte words, zero before the first call, written by nothing else) and a call
+// number `epoch` that differs from every earlier call's on this scratch and is never 0.
+inline size_t fma_code_words(int max_r) { return (size_t)2 * max_r > 4096 ? (size_t)2 * max_r : 4096; }
+cudaError_t fma_head(const bf16* h, const bf16* A, const bf16* B, int M, int mt, int d, int r, int V, int k, int mode,
+                     int32_t* ids, float* logprobs, float* logits, const Scratch& s, unsigned int epoch, int sm_count,
+                     cudaStream_t st);
 
 // ---- streaming path, three to sixteen rows (stream.cu) -----------------------------------
 struct StreamPlan {

@@ -23,7 +23,8 @@ constexpr size_t kRecWords = 68;                                                
 constexpr int kStaticParts = 320;
 constexpr size_t kPartBytes = (size_t)8 * kStaticParts * kRecWords * sizeof(float);  // [8 rows][320 records]
 constexpr size_t kCtlBytes = 256;                                                    // ticket, error word
-constexpr size_t kScratchBytes = kZBytes + kPartBytes + kCtlBytes;
+constexpr size_t kZqBytes = (size_t)2 * SLIMSPEC_STATIC_MAX_R * 8;                   // one- and two-row calls: the code as published (value, call number) words
+constexpr size_t kScratchBytes = kZBytes + kPartBytes + kCtlBytes + kZqBytes;
 
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
@@ -31,6 +32,7 @@ struct DeviceSetup {
     bool ready;
     unsigned char* base;     // device address of g_static_scratch on this device
     int sm_count;
+    unsigned int epoch;      // number of the last one- or two-row call on this device
 };
 constexpr int kMaxDevices = 64;
 DeviceSetup g_setup[kMaxDevices];
@@ -82,17 +84,27 @@ extern "C" int slimspec_head_topk_static(const void* h, const void* A, const voi
     s.part = reinterpret_cast<float*>(dev->base + kZBytes);
     s.tickets = reinterpret_cast<unsigned int*>(dev->base + kZBytes + kPartBytes);
     s.err = reinterpret_cast<int*>(dev->base + kZBytes + kPartBytes + 128);
+    s.zq = reinterpret_cast<uint2*>(dev->base + kZBytes + kPartBytes + kCtlBytes);
     s.max_parts = kStaticParts;
     cudaStream_t st = (cudaStream_t)stream;
     // The array keeps whatever the last call left; the ticket and the error word must start at 0.
     if (cudaMemsetAsync(dev->base + kZBytes + kPartBytes, 0, kCtlBytes, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
-    // the same choice of kernels as the context-based entry point: one or two rows, the FMA kernels
+    // the same choice of kernels as the context-based entry point: one or two rows, the FMA kernel
     const FmaPlan fp = fma_plan(M, d, r, V, k, dev->sm_count);
     cudaError_t e;
     if (fp.ok && fp.ncta <= kStaticParts) {
-        s.z = reinterpret_cast<float*>(dev->base);          // fp32 code, [r][mt]: it fits where the fragments would go
-        e = fma_downproj((const bf16*)h, (const bf16*)A, M, fp.mt, d, r, s, st);
-        if (e == cudaSuccess) e = fma_head(s.z, (const bf16*)B, M, fp.mt, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, st);
+        // the words of that area start as zeros (static storage) and only these calls write them; each call
+        // takes the next number, under the lock that also guards the set-up
+        unsigned int epoch;
+        {
+            std::lock_guard<std::mutex> lock(g_setup_mutex);
+            epoch = ++dev->epoch;
+            if (epoch == 0) {
+                if (cudaMemsetAsync(s.zq, 0, kZqBytes, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }
+                epoch = dev->epoch = 1;
+            }
+        }
+        e = fma_head((const bf16*)h, (const bf16*)A, (const bf16*)B, M, fp.mt, d, r, V, k, 0, out_ids, out_logprobs, nullptr, s, epoch, dev->sm_count, st);
     } else {
         e = stream_code((const bf16*)h, (const bf16*)A, M, d, r, V, k, s.zfrag, dev->sm_count, st);
         if (e == cudaSuccess) e = stream_head(s.zfrag, true, (const bf16*)B, M, r, V, k, 0, out_ids, out_logprobs, nullptr, s, dev->sm_count, true, nullptr, st);
