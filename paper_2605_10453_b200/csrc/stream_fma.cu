@@ -60,6 +60,7 @@ struct FmaParams {
     unsigned int* ticket;
     int* err;
     int pf_rows;          // rows of the slab asked into the L2 while waiting
+    int red_bytes;        // shared memory for the row groups' partial sums (at least what the merge needs)
 };
 
 __device__ __forceinline__ uint4 fma_ldg(const void* p)
@@ -75,13 +76,13 @@ __device__ __forceinline__ uint4 fma_ldg(const void* p)
 // word whole, old or new
 __device__ __forceinline__ void st_relaxed_gpu_u64(uint2* p, uint2 v)
 {
-    asm volatile("st.relaxed.gpu.global.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(v.x), "r"(v.y) : "memory");
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"((unsigned long long)v.x | ((unsigned long long)v.y << 32)) : "memory");
 }
 __device__ __forceinline__ uint2 ld_relaxed_gpu_u64(const uint2* p)
 {
-    uint2 v;
-    asm volatile("ld.relaxed.gpu.global.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p) : "memory");
-    return v;
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return make_uint2((uint32_t)v, (uint32_t)(v >> 32));
 }
 
 // ------------------------------------------------------------------------------------------
@@ -164,11 +165,11 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* cand = smem + kFmaEpFixed;                            // the epilogue's parked candidates
-    unsigned char* merge_area = cand + MT * kCand * 8;                   // the last CTA's merge
-    float* red = reinterpret_cast<float*>(merge_area + kFmaMergeBytes);  // [RG][MT][ct*8]; before that, the code jobs' warp sums
+    float* red = reinterpret_cast<float*>(cand + MT * kCand * 8);       // [RG][MT][ct*8]; before that, the code jobs' warp sums
+    unsigned char* merge_area = reinterpret_cast<unsigned char*>(red);   // the last CTA's merge, when the sums are no longer needed
     const int CT = p.ct, RG = p.rg;
     const int slab_cols = CT * 8;
-    float2* zs = reinterpret_cast<float2*>(red + (size_t)RG * MT * slab_cols);   // [kc][MT] (z, z) pairs
+    float2* zs = reinterpret_cast<float2*>(reinterpret_cast<unsigned char*>(red) + p.red_bytes);   // [kc][MT] (z, z) pairs
 
     const int tid = threadIdx.x;
     const int g = tid / CT, c = tid - g * CT;        // row group, column unit
@@ -329,7 +330,7 @@ static int fma_pick_mt(int M) { return M <= 1 ? 1 : 2; }
 
 struct FmaGeometry {
     int ncta, units_base, units_rem, max_units, ct, rg, u, kc, rec_words, threads;
-    int njobs, code_units, nsplit, job_rows;
+    int njobs, code_units, nsplit, job_rows, red_bytes;
     size_t smem;
 };
 
@@ -361,7 +362,8 @@ static bool fma_geometry(int mt, int d, int r, int V, int k, int sm_count, FmaGe
         if (g->kc < 1) return false;
     }
     g->rec_words = (2 + 2 * k + 3) / 4 * 4;
-    g->smem = (size_t)kFmaEpFixed + (size_t)mt * kCand * 8 + kFmaMergeBytes + (size_t)g->threads * mt * 32 + (size_t)g->kc * mt * 8;
+    g->red_bytes = g->threads * mt * 32 > kFmaMergeBytes ? g->threads * mt * 32 : kFmaMergeBytes;
+    g->smem = (size_t)kFmaEpFixed + (size_t)mt * kCand * 8 + g->red_bytes + (size_t)g->kc * mt * 8;
     if (g->smem > 200 * 1024) return false;
     // the down-projection's jobs: one 16-byte unit of A's columns each; the rows of A are split while
     // that leaves every CTA a job and a job at least a row per thread
@@ -420,7 +422,7 @@ cudaError_t fma_head(const bf16* h, const bf16* A, const bf16* B, int M, int mt,
     hp.ncta = g.ncta; hp.units_base = g.units_base; hp.units_rem = g.units_rem;
     hp.ct = g.ct; hp.rg = g.rg; hp.kc = g.kc; hp.rec_words = g.rec_words; hp.merge_inside = 1;
     hp.njobs = g.njobs; hp.code_units = g.code_units; hp.nsplit = g.nsplit; hp.job_rows = g.job_rows;
-    hp.zpart = s.zq; hp.epoch = epoch;
+    hp.zpart = s.zq; hp.epoch = epoch; hp.red_bytes = g.red_bytes;
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     {
