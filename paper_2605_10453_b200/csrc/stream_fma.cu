@@ -322,7 +322,7 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
         }
     }
     __syncthreads();
-    slab_epilogue<MT>(p, smem, cand, merge_area, red, RG, MT * slab_cols, slab_cols, my_units * 8, unit0 * 8);
+    slab_epilogue_few<MT>(p, smem, cand, merge_area, red, RG, MT * slab_cols, slab_cols, my_units * 8, unit0 * 8);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -352,6 +352,7 @@ static bool fma_geometry(int mt, int d, int r, int V, int k, int sm_count, FmaGe
     g->ct = (g->max_units + 31) / 32 * 32;
     g->rg = 512 / g->ct;
     if (g->rg > K) g->rg = K;
+    if (g->rg < 2) return false;      // the epilogue keeps at most four columns per thread
     g->threads = g->ct * g->rg;
     g->u = 16;
     // rows of the code per shared-memory chunk: all of K if it fits, else a multiple of rg*u
