@@ -14,6 +14,7 @@ struct slimspec_ctx {
     int forced_path;
     int last_path;
     long long launches;
+    unsigned int ticket_base;   // what the arrival counter will read when the next call starts
     unsigned int epoch;   // number of the last one- or two-row call (the code it publishes carries it)
     Scratch s;
     bf16* h_stage;        // device copy of host activations (head_topk_host)
@@ -73,6 +74,7 @@ extern "C" int slimspec_create(slimspec_ctx** out, int max_M, int max_d, int max
     c->sm_count = prop.multiProcessorCount;
     c->max_M = max_M; c->max_d = max_d; c->max_V = max_V; c->max_k = max_k;
     c->s.max_parts = kMaxParts;
+    c->s.ticket_base_host = &c->ticket_base;
     const size_t mpad = (size_t)round_up(max_M, kRowPad);
     const size_t z_elems = mpad * (size_t)max_d;
     // split-V records, padded to 16 bytes: the streaming path writes <= 16 rows x 320 records, the
@@ -163,6 +165,7 @@ extern "C" int slimspec_last_error(slimspec_ctx* c)
         cudaMemset(c->s.err, 0, sizeof(int));
         // tickets may have been left mid-count by the kernel that gave up
         cudaMemset(c->s.tickets, 0, 4096 * sizeof(unsigned int));
+        c->ticket_base = 0;
         return SLIMSPEC_ERR_TIMEOUT;
     }
     return SLIMSPEC_OK;

@@ -21,10 +21,17 @@ __device__ __forceinline__ unsigned int ticket_take(unsigned int* ticket)
     asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(ticket) : "memory");
     return old;
 }
+__device__ __forceinline__ unsigned int ld_acquire_gpu_u32(const unsigned int* p)
+{
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+static constexpr long long kArrivalPolls = 1ll << 22;      // reads of the counter before a merging CTA gives up (seconds)
 
 // ------------------------------------------------------------------------------------------
 // Step (4) of the epilogue and what follows it: a warp per row orders the parked candidates by counting
-// and writes the slab's record; then the arrival ticket, and the last CTA merges the records of every row.
+// and writes the slab's record; then the arrival ticket, and the last CTAs to arrive merge the records.
 template <int MT, class Params>
 __device__ __forceinline__ void slab_records(const Params& p, unsigned char* smem, unsigned char* scratch, unsigned char* merge_area,
     const float* lg, int ngroups, int gstride, int lpitch, int ncols, int col_base)
@@ -94,32 +101,43 @@ __device__ __forceinline__ void slab_records(const Params& p, unsigned char* sme
         }
     }
 
-    // ---- arrival: the last CTA merges the records of every row (many rows: a kernel of its own does,
-    // with two warps per row on as many SMs as it takes)
+    // ---- arrival.  The CTAs take tickets from a counter that only counts up (the call's first ticket is
+    // p.ticket_base).  The last R of them to arrive merge: each takes every R-th row, waits until the counter
+    // shows that all P have arrived (they are already running: it is a wait of a microsecond, bounded all
+    // the same), and runs two tasks per row, a warp each: the row's log-sum-exp, and its k best entries.
     if (!p.merge_inside) return;
     __syncthreads();
-    if (tid == 0) *s_ticket = ticket_take(p.ticket);
+    if (tid == 0) *s_ticket = ticket_take(p.ticket) - p.ticket_base;
     __syncthreads();
-    if (*s_ticket != (unsigned)(p.ncta - 1)) return;
-
-    // Two tasks per row, a warp each: the row's log-sum-exp, and its k best entries.
-    float* lse_s = reinterpret_cast<float*>(merge_area);                 // [16]
+    const int rows_at_once = max(1, nw >> 1);
+    const int R = min(P, (p.M + rows_at_once - 1) / rows_at_once);
+    const int me = (int)*s_ticket - (P - R);             // which of the R mergers this CTA is
+    if (me < 0) return;
+    if (me != R - 1) {
+        if (tid == 0) {
+            long long it = 0;
+            while (ld_acquire_gpu_u32(p.ticket) - p.ticket_base < (unsigned)P && ++it < kArrivalPolls) {}
+            if (it >= kArrivalPolls) atomicCAS(p.err, 0, ERR_WAIT_RECORD);
+        }
+        __syncthreads();
+    }
+    float* lse_s = reinterpret_cast<float*>(merge_area);                 // [16] by the CTA's own count of rows
     uint32_t* ok_all = reinterpret_cast<uint32_t*>(lse_s + 16);          // [16 rows][32] ordered keys
     int* oi_all = reinterpret_cast<int*>(ok_all + 16 * 32);              // [16 rows][32] their ids
     uint32_t* mk = reinterpret_cast<uint32_t*>(oi_all + 16 * 32) + warp * 2 * kMergeCand;     // this warp's candidates
     int* mi = reinterpret_cast<int*>(mk + kMergeCand);
-    for (int task = warp; task < 2 * p.M; task += nw) {
-        const int row = task >> 1;
-        if (P <= 5 * 32) merge_task<5>(p.part, P, RW, k, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
-        else merge_task<kMergeLists>(p.part, P, RW, k, row, task & 1, lane, lse_s, ok_all + row * 32, oi_all + row * 32, mk, mi, &cnt_s[warp]);
+    const int mine = (p.M - me + R - 1) / R;             // rows me, me + R, ...
+    for (int task = warp; task < 2 * mine; task += nw) {
+        const int lr = task >> 1, row = me + lr * R;
+        if (P <= 5 * 32) merge_task<5>(p.part, P, RW, k, row, task & 1, lane, lse_s + lr, ok_all + lr * 32, oi_all + lr * 32, mk, mi, &cnt_s[warp]);
+        else merge_task<kMergeLists>(p.part, P, RW, k, row, task & 1, lane, lse_s + lr, ok_all + lr * 32, oi_all + lr * 32, mk, mi, &cnt_s[warp]);
     }
     __syncthreads();
-    for (int e = tid; e < p.M * k; e += nt) {
-        const int row = e / k, j = e - row * k;
-        p.ids[e] = oi_all[row * 32 + j];
-        p.logprobs[e] = key2f(ok_all[row * 32 + j]) - lse_s[row];
+    for (int e = tid; e < mine * k; e += nt) {
+        const int lr = e / k, j = e - lr * k, row = me + lr * R;
+        p.ids[(size_t)row * k + j] = oi_all[lr * 32 + j];
+        p.logprobs[(size_t)row * k + j] = key2f(ok_all[lr * 32 + j]) - lse_s[lr];
     }
-    if (tid == 0) *p.ticket = 0;
 }
 
 // Epilogue of the head kernel.  The slab's logits lie in shared memory: logit (row, column c) is
@@ -128,8 +146,8 @@ __device__ __forceinline__ void slab_records(const Params& p, unsigned char* sme
 //   (1) maxima of groups of eight threads; (2) a warp per row: the k-th largest of these maxima
 //   bounds the slab's k-th largest logit from below; (3) sum of exp against the slab's maximum,
 //   logits that reach the bound are parked; (4) a warp per row orders the parked candidates by
-//   counting and writes the slab's record; then the arrival ticket, and the last CTA merges the
-//   records of every row the same way.
+//   counting and writes the slab's record; then the arrival ticket, and the last CTAs to arrive merge
+//   the records of every row the same way.
 // Nothing here depends on the order in which threads or CTAs arrive: results are reproducible.
 template <int MT, class Params>
 __device__ __forceinline__ void slab_epilogue(const Params& p, unsigned char* smem, unsigned char* scratch, unsigned char* merge_area,

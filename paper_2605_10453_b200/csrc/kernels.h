@@ -24,7 +24,8 @@ struct Scratch {
     uint32_t* thr0;      // tensor path: per-row starting bound of the top-k lists
     float* part;         // split-V partial records
     size_t part_elems;
-    unsigned int* tickets;  // arrival counters (self-resetting)
+    unsigned int* tickets;  // arrival counter: it only counts up
+    unsigned int* ticket_base_host;   // host: what the counter will read when the next call starts; a launcher that takes tickets adds its CTAs
     uint2* zq;              // one- and two-row path: the code as published (value, call number) words; no other path writes here
     int* err;            // device error word
     float* logits;       // generic path only: M x V fp32, grown on demand

@@ -86,6 +86,8 @@ extern "C" int slimspec_head_topk_static(const void* h, const void* A, const voi
     s.err = reinterpret_cast<int*>(dev->base + kZBytes + kPartBytes + 128);
     s.zq = reinterpret_cast<uint2*>(dev->base + kZBytes + kPartBytes + kCtlBytes);
     s.max_parts = kStaticParts;
+    unsigned int ticket_base = 0;           // the counter is cleared below, before every call
+    s.ticket_base_host = &ticket_base;
     cudaStream_t st = (cudaStream_t)stream;
     // The array keeps whatever the last call left; the ticket and the error word must start at 0.
     if (cudaMemsetAsync(dev->base + kZBytes + kPartBytes, 0, kCtlBytes, st) != cudaSuccess) { cudaGetLastError(); return SLIMSPEC_ERR_CUDA; }

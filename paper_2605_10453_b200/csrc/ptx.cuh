@@ -7,7 +7,7 @@
 namespace slimspec {
 
 // Device error codes written to the context's error word by a wait that ran out.
-enum : int { ERR_WAIT_FULL = 1, ERR_WAIT_EMPTY = 2, ERR_WAIT_ACC = 3, ERR_WAIT_FREE = 4 };
+enum : int { ERR_WAIT_FULL = 1, ERR_WAIT_EMPTY = 2, ERR_WAIT_ACC = 3, ERR_WAIT_FREE = 4, ERR_WAIT_RECORD = 5 };
 
 // Spin budget of one wait: ~0.25 s with the back-off below; a healthy wait takes microseconds.
 static constexpr uint32_t kSpinLimit = 1u << 22;

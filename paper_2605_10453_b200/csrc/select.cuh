@@ -101,11 +101,11 @@ __device__ __forceinline__ bool better(uint32_t ka, int ia, uint32_t kb, int ib)
 
 // ------------------------------------------------------------------------------------------
 // ------------------------------------------------------------------------------------------
-// One task of the last CTA's merge, run by one warp: kind 0 = the row's log-sum-exp from the
-// records' (maximum, sum-exp) pairs, kind 1 = its k best entries.  A lane owns the records lane,
+// One task of the merge, run by one warp: kind 0 = the row's log-sum-exp from the records'
+// (maximum, sum-exp) pairs, written to *lse_out; kind 1 = its k best entries.  A lane owns the records lane,
 // lane + 32, ... (NL of them at most) and keeps what it loads in registers: one round trip to the L2.
 template <int NL>
-__device__ __forceinline__ void merge_task(const float* part, int P, int RW, int k, int row, int kind, int lane, float* lse_s,
+__device__ __forceinline__ void merge_task(const float* part, int P, int RW, int k, int row, int kind, int lane, float* lse_out,
                                            uint32_t* ok, int* oi, uint32_t* mk, int* mi, int* cnt)
 {
     const float* rows = part + (size_t)row * P * RW;
@@ -124,7 +124,7 @@ __device__ __forceinline__ void merge_task(const float* part, int P, int RW, int
 #pragma unroll
         for (int q = 0; q < NL; ++q) gs += ms[q].y * __expf(ms[q].x - gm);
         gs = warp_sum(gs);
-        if (lane == 0) lse_s[row] = gm + __logf(gs);
+        if (lane == 0) *lse_out = gm + __logf(gs);
         return;
     }
     // the first three entries of every record (words 2..7), then the bound: at least k entries

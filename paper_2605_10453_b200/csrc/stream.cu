@@ -46,9 +46,10 @@ struct HeadParams {
     float* logits;
     float* part;              // records [M][ncta * npass][rec_words]
     unsigned int* ticket;
+    unsigned int ticket_base; // what the counter read when the call began
     int* err;
     int wait_prev;            // 1: the code is written by the kernel launched just before (PDL)
-    int merge_inside;         // 1: the last CTA to arrive merges the records; 0: the merge kernel follows
+    int merge_inside;         // 1: the last CTAs to arrive merge the records; 0: raw logits, nothing to merge
 };
 
 // ------------------------------------------------------------------------------------------
@@ -693,7 +694,9 @@ cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int 
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
     hp.wait_prev = after_producer_kernel ? 1 : 0;
-    hp.merge_inside = (mode == 1 || M <= 7) ? 1 : 0;       // measured: from 8 rows on the merge kernel is faster (2 us at 8 rows)
+    hp.merge_inside = 1;
+    hp.ticket_base = 0;
+    if (mode == 0) hp.ticket_base = *s.ticket_base_host;
     const bool pdl = after_producer_kernel;
     cudaError_t e;
     {
@@ -706,9 +709,9 @@ cudaError_t stream_head(const uint32_t* zfrag, bool lowrank, const bf16* B, int 
         else
             e = g.nch == 1 ? launch_head(k_stream_head_mma<16, 1, 1>, hp, g, pdl, st) : launch_head(k_stream_head_mma<16, 1, 2>, hp, g, pdl, st);
     }
-    if (launches) *launches += hp.merge_inside ? 1 : 2;
-    if (e != cudaSuccess || hp.merge_inside) return e;
-    return merge_records(s.part, M, hp.ncta, hp.rec_words, k, ids, logprobs, st);
+    if (launches) *launches += 1;
+    if (e == cudaSuccess && mode == 0) *s.ticket_base_host += (unsigned int)hp.ncta;      // the tickets this launch will take
+    return e;
 }
 
 }  // namespace slimspec

@@ -58,6 +58,7 @@ struct FmaParams {
     float* logits;
     float* part;          // split-V records [M][ncta][rec_words]
     unsigned int* ticket;
+    unsigned int ticket_base;   // what the counter read when the call began
     int* err;
     int pf_rows;          // rows of the slab asked into the L2 while waiting
     int red_bytes;        // shared memory for the row groups' partial sums (at least what the merge needs)
@@ -426,6 +427,8 @@ cudaError_t fma_head(const bf16* h, const bf16* A, const bf16* B, int M, int mt,
     hp.zpart = s.zq; hp.epoch = epoch; hp.red_bytes = g.red_bytes;
     hp.ids = ids; hp.logprobs = logprobs; hp.logits = logits;
     hp.part = s.part; hp.ticket = s.tickets; hp.err = s.err;
+    hp.ticket_base = 0;
+    if (mode == 0) hp.ticket_base = *s.ticket_base_host;
     {
         const size_t row_bytes = (size_t)g.max_units * 16 * g.ncta;      // one row of every slab
         const size_t rows = row_bytes ? kFmaPrefetchBytes / row_bytes : 0;
@@ -441,8 +444,9 @@ cudaError_t fma_head(const bf16* h, const bf16* A, const bf16* B, int M, int mt,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (mt == 1) return cudaLaunchKernelEx(&cfg, k_fma_head<1, 16>, hp);
-    return cudaLaunchKernelEx(&cfg, k_fma_head<2, 16>, hp);
+    const cudaError_t e = mt == 1 ? cudaLaunchKernelEx(&cfg, k_fma_head<1, 16>, hp) : cudaLaunchKernelEx(&cfg, k_fma_head<2, 16>, hp);
+    if (e == cudaSuccess && mode == 0) *s.ticket_base_host += (unsigned int)hp.ncta;      // the tickets this launch will take
+    return e;
 }
 
 }  // namespace slimspec

@@ -474,8 +474,8 @@ __global__ void __launch_bounds__(128) k_tc_merge(const float* __restrict__ part
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r2 = warp >> 1, row = blockIdx.x * 2 + r2;
     if (row < M) {
-        if (P <= 5 * 32) merge_task<5>(part, P, RW, k, row, warp & 1, lane, lse_s - row + r2, ok_s[r2], oi_s[r2], mk_s[warp], mi_s[warp], &cnt_s[warp]);
-        else merge_task<kMergeLists>(part, P, RW, k, row, warp & 1, lane, lse_s - row + r2, ok_s[r2], oi_s[r2], mk_s[warp], mi_s[warp], &cnt_s[warp]);
+        if (P <= 5 * 32) merge_task<5>(part, P, RW, k, row, warp & 1, lane, &lse_s[r2], ok_s[r2], oi_s[r2], mk_s[warp], mi_s[warp], &cnt_s[warp]);
+        else merge_task<kMergeLists>(part, P, RW, k, row, warp & 1, lane, &lse_s[r2], ok_s[r2], oi_s[r2], mk_s[warp], mi_s[warp], &cnt_s[warp]);
     }
     __syncthreads();
     if ((warp & 1) == 0 && row < M && lane < k) {
