@@ -157,7 +157,7 @@ int slimspec_kernel_timing_read(slimspec_ctx* ctx, double* total_ms, long long* 
  * driver allocations on its worker threads, or in a latency-critical section that cannot take
  * the device-wide synchronisation an allocation implies.  This call needs no context and calls
  * no allocating routine: its scratch (the fp32 code z, the per-slab records, a ticket and an
- * error word, about 1.4 MB) is a fixed device array inside the library image, held by every
+ * error word, about 1.5 MB) is a fixed device array inside the library image, held by every
  * GPU that loads the library until the process exits.
  *
  * Limits, because that array has a fixed size: M <= SLIMSPEC_STATIC_MAX_M,

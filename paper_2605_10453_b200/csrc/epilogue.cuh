@@ -277,7 +277,7 @@ __device__ __forceinline__ void slab_epilogue_few(const Params& p, unsigned char
             for (int c = tid; c < ncols; c += nt) p.logits[(size_t)row * p.V + col_base + c] = logit(row, c);
         return;
     }
-    static_assert(MT <= 2, "rows held in registers");
+    static_assert(MT <= 4, "rows held in registers");
     float x[MT][4];
 #pragma unroll
     for (int m = 0; m < MT; ++m)

@@ -43,7 +43,7 @@ cudaError_t generic_softmax_topk(const float* logits, int M, int V, int k, int32
 // ---- streaming path, one or two rows (stream_fma.cu) ------------------------------------
 struct FmaPlan {
     int ok;          // 0: shapes not supported by this kernel
-    int mt;          // rows per launch (1 or 2)
+    int mt;          // rows per launch (1, 2 or 4)
     int ncta;        // V slabs = CTAs
     int launches;    // kernels per call
 };
@@ -54,7 +54,7 @@ cudaError_t fma_prepare();
 // mode 0: fused log-softmax/top-k into ids/logprobs, mode 1: raw logits out.  Uses s.zq
 // (fma_code_words(max r) 8-byte words, zero before the first call, written by nothing else) and a call
 // number `epoch` that differs from every earlier call's on this scratch and is never 0.
-inline size_t fma_code_words(int max_r) { return (size_t)2 * max_r > 4096 ? (size_t)2 * max_r : 4096; }
+inline size_t fma_code_words(int max_r) { return (size_t)4 * max_r > 8192 ? (size_t)4 * max_r : 8192; }
 cudaError_t fma_head(const bf16* h, const bf16* A, const bf16* B, int M, int mt, int d, int r, int V, int k, int mode,
                      int32_t* ids, float* logprobs, float* logits, const Scratch& s, unsigned int epoch, int sm_count,
                      cudaStream_t st);

@@ -23,7 +23,7 @@ constexpr size_t kRecWords = 68;                                                
 constexpr int kStaticParts = 320;
 constexpr size_t kPartBytes = (size_t)8 * kStaticParts * kRecWords * sizeof(float);  // [8 rows][320 records]
 constexpr size_t kCtlBytes = 256;                                                    // ticket, error word
-constexpr size_t kZqBytes = (size_t)2 * SLIMSPEC_STATIC_MAX_R * 8;                   // one- and two-row calls: the code as published (value, call number) words
+constexpr size_t kZqBytes = (size_t)4 * SLIMSPEC_STATIC_MAX_R * 8;                   // one- and two-row calls: the code as published (value, call number) words
 constexpr size_t kScratchBytes = kZBytes + kPartBytes + kCtlBytes + kZqBytes;
 
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];

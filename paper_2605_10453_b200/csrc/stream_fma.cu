@@ -25,7 +25,11 @@ static constexpr int kFmaMaxColThreads = 256;   // threads across a slab's colum
 static constexpr int kFmaMaxCtas = 256;         // most slabs
 static constexpr int kFmaZChunkBytes = 64 * 1024;   // shared memory for the code, as (z, z) pairs
 static constexpr int kFmaEpFixed = (kEpFixedBytes + 127) / 128 * 128;      // the epilogue's fixed area
-static constexpr int kFmaMergeBytes = (16 + 2 * 16 * 32 + 4 * 2 * kMergeCand) * 4 + 64;   // the last CTA's merge: up to four tasks
+static constexpr int kFmaMergeBytes = (16 + 2 * 16 * 32 + 8 * 2 * kMergeCand) * 4 + 64;   // the last CTA's merge: up to eight tasks
+#ifndef SLIMSPEC_FMA4_MIN_A
+#define SLIMSPEC_FMA4_MIN_A (4u << 20)
+#endif
+static constexpr size_t kFmaFourRowsMinA = SLIMSPEC_FMA4_MIN_A;      // elements of A from which three and four rows take this kernel
 static constexpr int kFmaHelpAfter = 256;       // polls of the published code before a CTA computes the missing jobs itself
 
 // Bytes of the weight matrix (all CTAs together) the kernel asks into the L2 while it waits
@@ -112,7 +116,8 @@ __device__ __forceinline__ void fma_code_job(const FmaParams& p, int j, float* w
         for (int jj = 0; jj < 4; ++jj)
             a[jj] = (i0 + jj < rend) ? fma_ldg(Ac + (size_t)(i0 + jj) * p.K) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
-        for (int m = 0; m < MT; ++m) hv[m] = __ldcg(reinterpret_cast<const uint2*>(p.h + (size_t)m * p.d + i0));   // d is a multiple of 4
+        for (int m = 0; m < MT; ++m)     // d is a multiple of 4; with one and two rows MT = M
+            hv[m] = (MT <= 2 || m < p.M) ? __ldcg(reinterpret_cast<const uint2*>(p.h + (size_t)m * p.d + i0)) : make_uint2(0u, 0u);
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj) {
             const uint32_t w[4] = {a[jj].x, a[jj].y, a[jj].z, a[jj].w};
@@ -300,7 +305,7 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
         } else {
             for (int e = tid; e < (kend - kc0) * MT; e += blockDim.x) {
                 const int i = e / MT, m = e - i * MT;
-                const float zv = __bfloat162float(p.h[(size_t)m * p.d + kc0 + i]);
+                const float zv = (MT <= 2 || m < p.M) ? __bfloat162float(p.h[(size_t)m * p.d + kc0 + i]) : 0.f;
                 zs[e] = make_float2(zv, zv);
             }
         }
@@ -327,7 +332,7 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
 }
 
 // ------------------------------------------------------------------------------------------
-static int fma_pick_mt(int M) { return M <= 1 ? 1 : 2; }
+static int fma_pick_mt(int M) { return M <= 2 ? M : 4; }
 
 struct FmaGeometry {
     int ncta, units_base, units_rem, max_units, ct, rg, u, kc, rec_words, threads;
@@ -355,7 +360,7 @@ static bool fma_geometry(int mt, int d, int r, int V, int k, int sm_count, FmaGe
     if (g->rg > K) g->rg = K;
     if (g->rg < 2) return false;      // the epilogue keeps at most four columns per thread
     g->threads = g->ct * g->rg;
-    g->u = 16;
+    g->u = mt == 4 ? 8 : 16;      // loads a thread keeps in flight: the registers of four rows leave room for eight
     // rows of the code per shared-memory chunk: all of K if it fits, else a multiple of rg*u
     const int kc_max = kFmaZChunkBytes / (mt * 8);
     if (K <= kc_max) g->kc = K;
@@ -387,7 +392,9 @@ static bool fma_geometry(int mt, int d, int r, int V, int k, int sm_count, FmaGe
 FmaPlan fma_plan(int M, int d, int r, int V, int k, int sm_count)
 {
     FmaPlan sp = {0, 0, 0, 0};
-    if (M < 1 || M > 2) return sp;
+    // three and four rows only where A is large: there the down-projection inside this kernel, on all SMs,
+    // beats the other path's separate kernel (d = 8192: 8 to 32 MB of A); on the smaller heads the two are equal
+    if (M < 1 || M > 4 || (M > 2 && (r <= 0 || (size_t)d * r < kFmaFourRowsMinA))) return sp;
     const int mt = fma_pick_mt(M);
     FmaGeometry g;
     if (!fma_geometry(mt, d, r, V, k, sm_count, &g)) return sp;
@@ -404,6 +411,7 @@ cudaError_t fma_prepare()
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(k_fma_head<1, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess) return e;
     if ((e = cudaFuncSetAttribute(k_fma_head<2, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(k_fma_head<4, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess) return e;
     return cudaSuccess;
 }
 
@@ -444,7 +452,8 @@ cudaError_t fma_head(const bf16* h, const bf16* A, const bf16* B, int M, int mt,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = mt == 1 ? cudaLaunchKernelEx(&cfg, k_fma_head<1, 16>, hp) : cudaLaunchKernelEx(&cfg, k_fma_head<2, 16>, hp);
+    const cudaError_t e = mt == 1 ? cudaLaunchKernelEx(&cfg, k_fma_head<1, 16>, hp)
+                        : mt == 2 ? cudaLaunchKernelEx(&cfg, k_fma_head<2, 16>, hp) : cudaLaunchKernelEx(&cfg, k_fma_head<4, 8>, hp);
     if (e == cudaSuccess && mode == 0) *s.ticket_base_host += (unsigned int)hp.ncta;      // the tickets this launch will take
     return e;
 }

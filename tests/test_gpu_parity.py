@@ -87,6 +87,38 @@ def test_stream_path_matches_oracle(ctx, M, d, r, V, k):
     assert np.max(np.abs(lp - lp3)) < 1e-3
 
 
+def test_interleaved_shapes_share_the_scratch(ctx):
+    """One context, calls of changing shape and row count back to back without a synchronisation in
+    between: the one-launch kernel of one and two rows hands its code over through words in the
+    context's scratch that carry the number of the call, and every streaming kernel counts its CTAs
+    in on a counter that only counts up; neither may take a previous call's leftovers for its own."""
+    cases = [(1, 256, 64, 8 * 149, 10), (2, 512, 128, 8 * 1337, 7), (5, 96, 64, 8 * 777, 3), (1, 64, 64, 8 * 100, 10),
+             (16, 512, 64, 8 * 1501, 10), (2, 64, 64, 8 * 100, 5), (1, 512, 128, 8 * 1337, 7), (9, 256, 64, 8 * 149, 4)]
+    ctx.force_path(binding.PATH_STREAM)
+    inputs = [synth.make_inputs(M, d, r, V, seed=40 + i) for i, (M, d, r, V, k) in enumerate(cases)]
+    gpu = [dev(x) for x in inputs]
+    outs = []
+    for rep in range(3):
+        outs = []
+        for (M, d, r, V, k), g in zip(cases, gpu):
+            outs.append(ctx.slimspec_head_topk(g["h"], g["A"], g["B"], k))
+    torch.cuda.synchronize()
+    assert ctx.last_error() == binding.OK
+    for (M, d, r, V, k), x, (ids, lp) in zip(cases, inputs, outs):
+        b = obits(x)
+        st = check_topk(oracle.head_topk(b["h"], b["A"], b["B"], k), ids.cpu().numpy(), lp.cpu().numpy())
+        assert st["max_lp_err"] < 1e-3, (M, d, r, V, k)
+    # the full-rank head of one and two rows goes through the same kernel (its code is h itself)
+    for M in (1, 2):
+        h = synth.make_h(M, 256, 9)
+        W = synth.make_W(256, 8 * 901, 9)
+        ids, lp = ctx.fullhead_topk(h.to(DEV), W.to(DEV), 6)
+        torch.cuda.synchronize()
+        st = check_topk(oracle.fullhead_topk(oracle.bf16_bits(h), oracle.bf16_bits(W), 6), ids.cpu().numpy(), lp.cpu().numpy())
+        assert st["max_lp_err"] < 1e-3
+    ctx.force_path(binding.PATH_AUTO)
+
+
 TENSOR_SHAPES = [
     # M, d, r, V, k -- one and several row blocks, ragged last column tile, V below one tile
     (1, 64, 64, 64, 3),
