@@ -467,7 +467,7 @@ __global__ void __launch_bounds__(256, 2) k_stream_head_mma(const HeadParams p) 
         }
     __syncthreads();
     unsigned char* lists = reinterpret_cast<unsigned char*>(lg + (size_t)MT * lpitch);
-    slab_epilogue<MT>(p, smem, lists, zarea, lg, 1, 0, lpitch, my_units * 8, unit0 * 8);
+    slab_epilogue_rows<MT>(p, smem, lists, zarea, lg, lpitch, my_units * 8, unit0 * 8);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -69,6 +69,8 @@ STREAM_SHAPES = [
     (8, 1024, 128, 8 * 2500, 10),
     (7, 160, 320, 8 * 148 * 130, 5),      # 130 units per slab: two column passes
     (11, 512, 64, 8 * 1501, 10),          # two row tiles (8 + 3)
+    (3, 8192, 512, 8 * 1501, 10),         # a large A: three and four rows take the one-launch kernel
+    (4, 4096, 1024, 8 * 777, 5),
 ]
 
 
