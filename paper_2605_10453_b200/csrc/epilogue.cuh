@@ -181,7 +181,7 @@ __device__ __forceinline__ void slab_epilogue_rows(const Params& p, unsigned cha
         float lm = -FLT_MAX;
         for (int c = lane; c < ncols; c += 32) lm = fmaxf(lm, lr[c] + 0.f);       // -0 becomes +0: keys and float compares then agree
         const uint32_t lk = f2key(lm);
-        const uint32_t kth = warp_kth_largest_any(lk, min(k, 32), lane);
+        const uint32_t kth = warp_kth_largest(lk, min(k, 32), lane);       // a lone warp waits on latencies: 32 independent shuffles beat k dependent rounds
         const float cm = key2f(warp_max_u32(lk));
         float s = 0.f;
         int n = 0;
