@@ -21,8 +21,12 @@
 
 namespace slimspec {
 
-static constexpr int kMmaWarps = 7;                   // warps of a CTA of the tensor-core kernel (two CTAs per SM): 64 columns each
-static constexpr int kMmaThreads = kMmaWarps * 32;
+static constexpr int kMmaWarps = 7;                   // warps of a CTA of the tensor-core kernel (two CTAs per SM): 64 columns each;
+                                                      // eight where that saves the epilogue a round of rows (see mma_warps)
+// The epilogue gives each row to one warp: 8 rows on 7 warps take two rounds, 16 rows three.  An eighth
+// warp (idle in the stream when the slab has no columns for it) saves a round there: M = 8: 41.1 -> 39.6 us,
+// M = 16: 48.1 -> 46.4 us; with other row counts it only adds a party to the barriers (+0.4 to 0.7 us).
+static int mma_warps(int M) { return (M == 8 || M >= 15) ? 8 : kMmaWarps; }
 static constexpr size_t kMmaSmem = 76 * 1024;         // its shared memory: two such CTAs and the down-projection's CTA of the next call share an SM
 static constexpr int kMaxStages = 8;                  // most stages of the shared-memory ring
 enum : int { kCodePacked = 1, kCodeSplit = 2, kCodePlain = 3, kCodeRows = 4 };
@@ -473,7 +477,7 @@ __global__ void __launch_bounds__(256, 2) k_stream_head_mma(const HeadParams p) 
 // ------------------------------------------------------------------------------------------
 struct Geometry {
     int ncta, units_base, units_rem, rec_words;
-    int nch, pitch_units, ns, nkb, kb_chunk, nchunks;
+    int nch, pitch_units, ns, nkb, kb_chunk, nchunks, warps;
     size_t zarea_bytes, smem;
 };
 
@@ -497,7 +501,8 @@ static bool geometry(int M, int zparts, int K, int V, int k, int sm_count, Geome
     g->units_base = units / ncta;
     g->units_rem = units % ncta;
     const int mma_units = g->units_base + (g->units_rem ? 1 : 0);
-    g->nch = (mma_units + 8 * kMmaWarps - 1) / (8 * kMmaWarps);
+    g->warps = mma_warps(M);
+    g->nch = (mma_units + 8 * g->warps - 1) / (8 * g->warps);
     if (g->nch > 2) return false;
     g->pitch_units = mma_units | 1;
     g->nkb = (K + 15) / 16;
@@ -683,7 +688,7 @@ static cudaError_t launch_head(Kern kern, const HeadParams& hp, const Geometry& 
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(hp.ncta);
-    cfg.blockDim = dim3(kMmaThreads);
+    cfg.blockDim = dim3(g.warps * 32);
     cfg.dynamicSmemBytes = g.smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
