@@ -97,7 +97,7 @@ __device__ __forceinline__ uint2 ld_relaxed_gpu_u64(const uint2* p)
 // keeps), the warps meet in shared memory.  Sums run in a fixed order, so whoever computes a job
 // -- its owner or a helper -- publishes the same bits.
 template <int MT>
-__device__ __forceinline__ void fma_code_job(const FmaParams& p, int j, float* wpart)
+__device__ __forceinline__ void fma_code_job(const FmaParams& p, int j, float* wpart, const uint4 (&apre)[4], bool have_pre)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nt = blockDim.x, nw = nt >> 5;
     const int s = j / p.code_units, u = j - s * p.code_units;
@@ -112,9 +112,11 @@ __device__ __forceinline__ void fma_code_job(const FmaParams& p, int j, float* w
     for (int i0 = rbeg + tid * 4; i0 < rend; i0 += nt * 4) {
         uint4 a[4];
         uint2 hv[MT];
+        // the first four rows of the CTA's own job were sent for before the wait (weights may be)
+        const bool pre = have_pre && i0 == rbeg + tid * 4;
 #pragma unroll
         for (int jj = 0; jj < 4; ++jj)
-            a[jj] = (i0 + jj < rend) ? fma_ldg(Ac + (size_t)(i0 + jj) * p.K) : make_uint4(0u, 0u, 0u, 0u);
+            a[jj] = pre ? apre[jj] : (i0 + jj < rend) ? fma_ldg(Ac + (size_t)(i0 + jj) * p.K) : make_uint4(0u, 0u, 0u, 0u);
 #pragma unroll
         for (int m = 0; m < MT; ++m)     // d is a multiple of 4; with one and two rows MT = M
             hv[m] = (MT <= 2 || m < p.M) ? __ldcg(reinterpret_cast<const uint2*>(p.h + (size_t)m * p.d + i0)) : make_uint2(0u, 0u);
@@ -199,6 +201,22 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
     const bool active = c < my_units;
     const bf16* base = p.B + (size_t)(unit0 + c) * 8;
 
+    // the CTA's own job of the down-projection: its first four rows of A per thread go out now,
+    // ahead of everything else, so that after the wait only h is missing
+    uint4 apre[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) apre[jj] = make_uint4(0u, 0u, 0u, 0u);
+    const bool have_pre = lowrank && cta < p.njobs;
+    if (have_pre) {
+        const int s = cta / p.code_units, u = cta - s * p.code_units;
+        const int rbeg = s * p.job_rows, rend = min(p.d, rbeg + p.job_rows);
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+            const int i = rbeg + tid * 4 + jj;
+            if (i < rend) apre[jj] = fma_ldg(p.A + (size_t)i * K + u * 8);
+        }
+    }
+
     // Two sets of UH loads each: one set is consumed while the other is in flight, so a wait
     // for the older set never waits for loads issued after it.
     constexpr int UH = U / 2;
@@ -233,7 +251,7 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
 
     // ---- this CTA's jobs of the down-projection
     if (lowrank)
-        for (int j = cta; j < p.njobs; j += p.ncta) fma_code_job<MT>(p, j, red);
+        for (int j = cta; j < p.njobs; j += p.ncta) fma_code_job<MT>(p, j, red, apre, have_pre && j == cta);
 
     float2 acc[MT][4];
 #pragma unroll
@@ -298,7 +316,7 @@ __global__ void __launch_bounds__(512, 1) k_fma_head(const FmaParams p)
                     for (int j = 0; j < p.njobs; ++j) {
                         const int s = j / p.code_units, u = j - s * p.code_units;
                         const bool missing = ld_relaxed_gpu_u64(p.zpart + ((size_t)s * K + u * 8) * MT).y != p.epoch;
-                        if (__syncthreads_or(missing)) fma_code_job<MT>(p, j, red);
+                        if (__syncthreads_or(missing)) fma_code_job<MT>(p, j, red, apre, false);
                     }
                 }
             }
