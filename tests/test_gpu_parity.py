@@ -121,6 +121,34 @@ def test_interleaved_shapes_share_the_scratch(ctx):
     ctx.force_path(binding.PATH_AUTO)
 
 
+def test_random_shapes_in_batches_against_oracle(ctx):
+    """Seeded random shapes (rows 1..16, every streaming kernel and its variants by row count), enqueued six
+    at a time without a synchronisation in between, twice over; every result against the oracle."""
+    import random
+    rng = random.Random(20260510)
+    ctx.force_path(binding.PATH_AUTO)
+    batch = []
+    for it in range(24):
+        M = rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 12, 15, 16])
+        d = rng.choice([64, 128, 256, 520, 1024, 2048, 4096])
+        r = rng.choice([16, 32, 64, 128, 256, 512])
+        V = 8 * rng.randint(20, 2000)
+        k = rng.randint(1, min(32, V))
+        x = synth.make_inputs(M, d, r, V, seed=100 + it)
+        batch.append((M, d, r, V, k, x, dev(x)))
+        if len(batch) < 6:
+            continue
+        for rep in range(2):
+            outs = [ctx.slimspec_head_topk(g["h"], g["A"], g["B"], k_) for (_, _, _, _, k_, _, g) in batch]
+        torch.cuda.synchronize()
+        assert ctx.last_error() == binding.OK
+        for (M_, d_, r_, V_, k_, x_, _), (ids, lp) in zip(batch, outs):
+            b = obits(x_)
+            st = check_topk(oracle.head_topk(b["h"], b["A"], b["B"], k_), ids.cpu().numpy(), lp.cpu().numpy())
+            assert st["max_lp_err"] < 1e-3, (M_, d_, r_, V_, k_)
+        batch = []
+
+
 TENSOR_SHAPES = [
     # M, d, r, V, k -- one and several row blocks, ragged last column tile, V below one tile
     (1, 64, 64, 64, 3),
